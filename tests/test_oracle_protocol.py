@@ -1,0 +1,360 @@
+"""Pins for the protocol oracle against what the paper and mathematics fix (CPU only)."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import protocol as op
+from paper_1902_01064_b200 import inputs
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden", "paper_examples.txt")
+STUCK = 10 ** 15
+
+
+def golden():
+    out = {}
+    for line in open(GOLD):
+        line = line.split("#")[0].strip()
+        if "=" in line:
+            k, v = line.split("=", 1)
+            out[k.strip()] = v.strip()
+    return out
+
+
+def rand_ticks(rng, N, iters, lo=1, hi=6):
+    return rng.integers(lo, hi, size=(N, iters)).astype(np.uint64)
+
+
+GRAPHS = [("ring6", inputs.ring(6)), ("cycle5", inputs.directed_cycle(5)), ("torus", inputs.torus(3, 3)),
+          ("complete4", inputs.complete(4)), ("ringbased8", inputs.ring_based(8))]
+
+
+# ------------------------------------------------------------------ Theorem 1
+@pytest.mark.parametrize("name,n_in", GRAPHS)
+def test_theorem1_gap_bounded_by_shortest_path(name, n_in):
+    rng = np.random.default_rng(1)
+    N = len(n_in)
+    dist = op.shortest_paths(n_in)
+    for trial in range(10):
+        seen = []
+
+        def chk(p):
+            for i in range(N):
+                for j in range(N):
+                    assert p.Iter[i] - p.Iter[j] <= dist[j][i]
+            seen.append(max(p.Iter) - min(p.Iter))
+        op.simulate(n_in, rand_ticks(rng, N, 12, 1, 9), 12, on_round=chk)
+        assert seen
+
+
+def test_theorem1_bound_is_reached_on_a_chain():
+    # Chain 0 -> 1 -> 2 -> 3 with a slow head: the worker at distance d from worker 0 gets exactly
+    # d iterations ahead of it, so the bound of Theorem 1 is tight.
+    n_in = [[0], [0, 1], [1, 2], [2, 3]]
+    ticks = np.ones((4, 8), np.uint64)
+    ticks[0, :] = 100
+    best = [0] * 4
+
+    def chk(p):
+        for i in range(4):
+            best[i] = max(best[i], p.Iter[i] - p.Iter[0])
+    op.simulate(n_in, ticks, 8, on_round=chk)
+    assert best == [0, 1, 2, 3]
+
+
+# ------------------------------------------------------------------ closed form (max-plus recurrence)
+def recurrence(n_in, T, iters, s, max_ig):
+    """start/finish times for b = 0, no skipping: a worker finishes Recv(k) once its compute is over
+    and every in-neighbour has entered iteration k - s; it enters k+1 once every out-neighbour has
+    entered k + 1 - max_ig."""
+    N = len(n_in)
+    n_out = [[i for i in range(N) if j in n_in[i] and i != j] for j in range(N)]
+    start = np.zeros((N, iters + 1), np.int64)
+    fin = np.zeros((N, iters), np.int64)
+    for k in range(iters):
+        for i in range(N):
+            f = start[i, k] + int(T[i][k])
+            for j in n_in[i]:
+                if j != i:
+                    f = max(f, start[j, max(k - s, 0)])
+            fin[i, k] = f
+        for i in range(N):
+            st = fin[i, k]
+            if max_ig is not None and k + 1 - max_ig >= 0:
+                for j in n_out[i]:
+                    st = max(st, start[j, k + 1 - max_ig])
+            start[i, k + 1] = st
+    return start, fin
+
+
+@pytest.mark.parametrize("s,max_ig", [(0, None), (0, 1), (0, 3), (2, None), (2, 2), (3, 1)])
+def test_times_and_versions_match_maxplus_recurrence(s, max_ig):
+    rng = np.random.default_rng(7 + s)
+    for name, n_in in GRAPHS:
+        N = len(n_in)
+        iters = 9
+        T = rng.integers(10 ** 6, 3 * 10 ** 6, size=(N, iters)).astype(np.uint64)
+        if max_ig is not None and max_ig < 1:
+            continue
+        starts = {}
+
+        def chk(p):
+            for i in range(N):
+                starts.setdefault((i, p.Iter[i]), p.now)
+        tr = op.simulate(n_in, T, iters, s=s, b=0, max_ig=max_ig, weight_mode=op.STALE_LINEAR, on_round=chk)
+        # every wait looks at a lower or equal level whose start time is already final, so one
+        # sweep per level evaluates the recurrence
+        st, fin = recurrence(n_in, T, iters, s, max_ig)
+        for i in range(N):
+            for k in range(1, iters):
+                assert starts[(i, k)] == st[i, k], (name, i, k)
+        assert tr.makespan == fin[:, iters - 1].max()
+        # generic position: consumed version = newest v <= k with start(j, v) <= finish(i, k)
+        for i in range(N):
+            for k in range(iters):
+                for (j, v, w) in tr.rec[(k, i)]:
+                    if j == i:
+                        assert v == k
+                        continue
+                    cand = [u for u in range(0, k + 1) if st[j, u] < fin[i, k]]
+                    ties = [u for u in range(0, k + 1) if st[j, u] == fin[i, k]]
+                    if not ties:
+                        assert v == max(cand), (name, i, k, j)
+                    assert k - s <= v <= k
+                    assert w == v - (k - s) + 1
+
+
+# ------------------------------------------------------------------ tokens
+@pytest.mark.parametrize("max_ig", [1, 2, 3])
+@pytest.mark.parametrize("name,n_in", GRAPHS)
+def test_token_identity_theorem2_and_capacity(name, n_in, max_ig):
+    rng = np.random.default_rng(3)
+    N = len(n_in)
+    dist = op.shortest_paths(n_in)
+    for trial in range(6):
+        def chk(p):
+            assert op.token_identity_holds(p)                    # Section 4.2 proof
+            for i in range(N):
+                for j in range(N):
+                    if i != j:
+                        assert p.Iter[i] - p.Iter[j] <= min(dist[j][i], max_ig * dist[i][j])   # Theorem 2
+            for (a, c), q in p.token_q.items():                  # TokenQ(a -> c): capacity bound
+                assert len(q) <= max_ig * (dist[a][c] + 1)
+        op.simulate(n_in, rand_ticks(rng, N, 10, 1, 12), 10, max_ig=max_ig, on_round=chk)
+
+
+def test_token_prose_example_sender_stops_at_max_ig():
+    g = golden()
+    max_ig = int(g["token_example.max_ig"])
+    # B (=1) sends to A (=0); A never finishes its first Compute.
+    n_in = [[0, 1], [1]]
+    ticks = np.ones((2, 10), np.uint64)
+    ticks[0, 0] = STUCK
+    top = [0]
+
+    def chk(p):
+        if p.Iter[0] == 0 and p.now < STUCK:
+            top[0] = max(top[0], p.Iter[1])
+    op.simulate(n_in, ticks, 10, max_ig=max_ig, on_round=chk)
+    assert top[0] == int(g["token_example.sender_final_iter"])
+    # without token queues nothing stops the sender (Theorem 1 only bounds the receiver)
+    top[0] = 0
+    op.simulate(n_in, ticks, 10, max_ig=None, on_round=chk)
+    assert top[0] == 9
+
+
+# ------------------------------------------------------------------ bounded staleness
+@pytest.mark.parametrize("s", [1, 2, 4])
+@pytest.mark.parametrize("name,n_in", GRAPHS)
+def test_staleness_window_and_gap(name, n_in, s):
+    rng = np.random.default_rng(11)
+    N = len(n_in)
+    dist = op.shortest_paths(n_in)
+    for trial in range(5):
+        def chk(p):
+            for i in range(N):
+                for j in range(N):
+                    if i != j:
+                        assert p.Iter[i] - p.Iter[j] <= (s + 1) * dist[j][i]      # Table 1, row 2
+        tr = op.simulate(n_in, rand_ticks(rng, N, 12, 1, 30), 12, s=s, weight_mode=op.STALE_LINEAR, on_round=chk)
+        for (k, i), rec in tr.rec.items():
+            assert sorted(j for j, _, _ in rec) == sorted(n_in[i])               # b = 0: everyone
+            for (j, v, w) in rec:
+                assert k - s <= v <= k                                           # never older than s
+                assert w == v - (k - s) + 1                                      # Eq. 2 numerator
+            assert tr.den[(k, i)] == sum(w for _, _, w in rec)
+
+
+def test_staleness_stuck_neighbour_reaches_s_plus_one():
+    g = golden()
+    s = int(g["staleness_example.s"])
+    n_in = inputs.complete(3)
+    ticks = np.ones((3, 12), np.uint64)
+    ticks[0, 0] = STUCK
+    lead = [0, 0, 0]
+
+    def chk(p):
+        if p.now < STUCK:
+            for i in range(3):
+                lead[i] = max(lead[i], p.Iter[i] - p.Iter[0])
+    op.simulate(n_in, ticks, 12, s=s, on_round=chk)
+    assert lead[1] == lead[2] == int(g["staleness_example.max_lead"]) == s + 1
+
+
+# ------------------------------------------------------------------ backup workers
+def test_backup_counts_and_versions():
+    rng = np.random.default_rng(5)
+    for name, n_in in GRAPHS:
+        N = len(n_in)
+        for b in (1, 2):
+            if any(b >= len(nb) for nb in n_in):
+                continue
+            tr = op.simulate(n_in, rand_ticks(rng, N, 10, 1, 40), 10, s=0, b=b, max_ig=2)
+            short = 0
+            for (k, i), rec in tr.rec.items():
+                d = len(n_in[i])
+                assert d - b <= len(rec) <= d                                     # Fig. alg4: needed + extras
+                assert all(v == k for _, v, _ in rec)                             # only iteration k
+                assert (i, k, 1) in rec                                           # own update, plain mean
+                assert tr.den[(k, i)] == len(rec)
+                short += len(rec) < d
+            assert short > 0, "backup never used: test is vacuous"
+
+
+def test_backup_prose_example_three_workers():
+    g = golden()
+    assert int(g["backup_example.workers"]) == 3
+    b = 2 - int(g["backup_example.needed_neighbour_updates"])                    # two neighbours, one needed
+    n_in = inputs.complete(3)
+    ticks = np.ones((3, 15), np.uint64)
+    ticks[0, 0] = STUCK
+    top = [0, 0, 0]
+
+    def chk(p):
+        if p.now < STUCK:
+            for i in range(3):
+                top[i] = max(top[i], p.Iter[i])
+    # no token queues: B and C run to the end relying on one another
+    op.simulate(n_in, ticks, 15, s=0, b=b, max_ig=None, on_round=chk)
+    assert top == [0, 14, 14]
+    # without backup they are dragged down: one iteration ahead at most (Theorem 1)
+    top[:] = [0, 0, 0]
+    op.simulate(n_in, ticks, 15, s=0, b=0, max_ig=None, on_round=chk)
+    assert top == [0, 1, 1]
+    # with token queues the unbounded gap is cut at max_ig (Section 4.3)
+    for max_ig in (1, 2, 4):
+        top[:] = [0, 0, 0]
+        op.simulate(n_in, ticks, 15, s=0, b=b, max_ig=max_ig, on_round=chk)
+        assert top == [0, max_ig, max_ig]
+
+
+@pytest.mark.parametrize("s,b", [(0, 1), (2, 0), (2, 1), (1, 2)])
+def test_table1_last_row_with_tokens(s, b):
+    rng = np.random.default_rng(13)
+    for name, n_in in GRAPHS:
+        if any(b >= len(nb) for nb in n_in):
+            continue
+        N = len(n_in)
+        dist = op.shortest_paths(n_in)
+        b0 = 10 ** 9 if b > 0 else s + 1
+        for max_ig in (1, 3):
+            def chk(p):
+                assert op.token_identity_holds(p)
+                for i in range(N):
+                    for j in range(N):
+                        if i != j:
+                            assert p.Iter[i] - p.Iter[j] <= min(b0 * dist[j][i], max_ig * dist[i][j])
+            tr = op.simulate(n_in, rand_ticks(rng, N, 10, 1, 25), 10, s=s, b=b, max_ig=max_ig,
+                             weight_mode=op.STALE_LINEAR, on_round=chk)
+            for (k, i), rec in tr.rec.items():
+                assert len(rec) >= len(n_in[i]) - b
+                assert all(k - s <= v <= k for _, v, _ in rec)
+
+
+# ------------------------------------------------------------------ skipping iterations
+def test_skipping_invariants_and_progress():
+    n_in = inputs.ring_based(8)
+    N, iters, s, max_ig = 8, 40, 3, 3
+    ticks = np.ones((N, iters), np.uint64)
+    ticks[2, :] = 4                                                # deterministic straggler (Section 7.3.5)
+    for max_skip in (1, 2, 4):
+        planned = []
+
+        def chk(p):
+            assert op.token_identity_holds(p)                      # (k - k0) tokens moved each way
+            for i in range(N):
+                if p.phase[i] == op._JUMPRECV:
+                    outs = [j for j in p.n_out[i] if j != i]
+                    # never jump past the slowest out-neighbour (Section 5: max_jump - max_ig)
+                    assert p.jump_to[i] <= min(p.Iter[j] for j in outs)
+                    assert 2 <= p.jump_to[i] - p.Iter[i] <= max_skip + 1
+                    planned.append((i, p.Iter[i], p.jump_to[i]))
+        tr = op.simulate(n_in, ticks, iters, s=s, max_ig=max_ig, max_skip=max_skip,
+                         weight_mode=op.STALE_LINEAR, on_round=chk)
+        base = op.simulate(n_in, ticks, iters, s=s, max_ig=max_ig, max_skip=0, weight_mode=op.STALE_LINEAR)
+        assert planned and all(i == 2 for i, _, _ in planned)      # only the straggler identifies itself
+        assert tr.makespan < base.makespan                         # others advance faster
+        A = tr.to_arrays()
+        for (i, k0, k) in set(planned):
+            assert A["op"][k - 1, i] == op.JUMP
+            assert all(A["op"][lv, i] == op.IDLE for lv in range(k0 + 1, k - 1))
+            rec = tr.rec[(k - 1, i)]
+            own = [r for r in rec if r[0] == i]
+            assert own == [(i, k0 + 1, s + 1)]                     # own parameters, weighted as iteration k-1
+            assert all((k - 1) - s <= v <= k - 1 for j, v, _ in rec if j != i)
+        # skipped iterations are never consumed by anyone
+        skipped = {(i, v) for (i, k0, k) in planned for v in range(k0 + 1, k)}
+        for (k, i), rec in tr.rec.items():
+            for (j, v, _) in rec:
+                if j != i:
+                    assert (j, v) not in skipped
+
+
+def test_skipping_needs_token_queues_and_stays_off_by_default():
+    n_in = inputs.ring(4)
+    ticks = np.ones((4, 6), np.uint64)
+    ticks[1, :] = 5
+    with pytest.raises(ValueError):
+        op.simulate(n_in, ticks, 6, s=1, max_ig=None, max_skip=1)
+    tr = op.simulate(n_in, ticks, 6, s=1, max_ig=1)
+    assert (tr.op == op.NORMAL).all()
+
+
+# ------------------------------------------------------------------ reductions to the standard algorithm
+def test_equal_speeds_reduce_to_standard_algorithm():
+    for name, n_in in GRAPHS:
+        N = len(n_in)
+        for (s, b, max_ig) in [(0, 0, None), (2, 0, 2), (0, 1, 1), (1, 1, 3)]:
+            if any(b >= len(nb) for nb in n_in):
+                continue
+            tr = op.simulate(n_in, np.full((N, 5), 3, np.uint64), 5, s=s, b=b, max_ig=max_ig,
+                             weight_mode=op.STALE_LINEAR)
+            for (k, i), rec in tr.rec.items():
+                assert [(j, v) for j, v, _ in rec] == [(j, k) for j in n_in[i]]   # Fig. alg0: all of iteration k
+                assert len(set(w for _, _, w in rec)) == 1                         # Eq. 2 == Eq. 1 here
+            assert tr.makespan == 15
+
+
+def test_weights_closed_forms():
+    nums, den = op.reduce_weights([7, 7, 7], 7, 3, op.UNIFORM)
+    assert (nums, den) == ([1, 1, 1], 3)                                           # Eq. 1: 1/|N_in|
+    nums, den = op.reduce_weights([7, 6, 4, 5], 7, 3, op.STALE_LINEAR)
+    assert (nums, den) == ([4, 3, 1, 2], 10)                                       # Eq. 2, k - s = 4
+    for s in range(5):
+        nums, den = op.reduce_weights([9] * 4, 9, s, op.STALE_LINEAR)
+        assert all(n * 4 == den for n in nums)                                     # all fresh -> uniform
+
+
+def test_rejects_bad_graphs():
+    with pytest.raises(ValueError):
+        op.simulate([[1], [0, 1]], np.ones((2, 2), np.uint64), 2)
+    with pytest.raises(ValueError):
+        op.simulate(inputs.ring(4), np.ones((4, 2), np.uint64), 2, b=3)
+
+
+def test_deadlock_is_reported():
+    class NoTokens(op.HopProtocol):
+        def _tokens_available(self, i, n):
+            return False
+    with pytest.raises(op.Deadlock):
+        NoTokens(inputs.ring(4), np.ones((4, 3), np.uint64), 3, max_ig=1).run()
