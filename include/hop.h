@@ -1,0 +1,190 @@
+/*
+ * hop.h -- C ABI of the Hop hot path (heterogeneity-aware decentralized SGD, arXiv 1902.01064)
+ * for N simulated workers whose parameter replicas all live in one GPU's memory.
+ *
+ * One logical iteration ("level" k) for all workers is: every worker i that executes iteration k
+ * computes a minibatch gradient on x_{k,i} (Fig. alg0 step 1; the "parallel approach" of
+ * Section 3.2: the gradient is taken before the Reduce), averages the in-neighbour versions the
+ * queue protocol let it consume (Recv/Reduce of Fig. alg4 and Fig. alg3, weights of Eq. 1 or
+ * Eq. 2) and applies the gradient (Fig. alg0 step 3).  Which (in-neighbour, version) pairs are
+ * consumed is an integer "trace" produced on the host by a deterministic simulation of the
+ * protocol (update queues Section 4.1, token queues Section 4.2, backup workers Section 4.3,
+ * bounded staleness Section 4.4, skipping iterations Section 5).
+ *
+ * Conventions
+ *   - Every function returns 0 (HOP_OK) or a negative hop_status; hop_last_error() gives a
+ *     human-readable message for the last failure on that context (or of hop_create /
+ *     hop_trace_create when passed NULL).  Nothing throws, aborts or traps.
+ *   - "host" pointers are ordinary CPU memory, read or written before the call returns.
+ *     "device" pointers are CUDA device memory owned by the caller; the context only borrows
+ *     them and they must stay valid until hop_destroy or the next bind call.
+ *   - Work is enqueued on the CUDA stream given to hop_bind_buffers and is asynchronous unless
+ *     stated otherwise.  A context is not thread-safe.
+ *   - The library keeps small device tables of its own (the uploaded trace, per-minibatch hinge
+ *     coefficients); they are allocated in hop_load_trace / hop_bind_svm_* / hop_step_host and
+ *     freed in hop_destroy.  hop_step itself allocates nothing.
+ *   - There is no CPU fallback: device entry points fail with HOP_E_CUDA when no GPU is usable.
+ *
+ * Data layout in device memory (all float32, row-major, the parameter index fastest):
+ *   X[N][s+1][P]  ring of s+1 versions per worker; version v of worker i sits in slot v mod (s+1)
+ *                 (Section 6: one queue per iteration slot, index mod(iter, #queues)).
+ *   M[N][P]       momentum buffers (only with momentum != 0)
+ *   G[N][P]       dense gradients of the current level (not used by the CSR SVM mode)
+ */
+#ifndef HOP_B200_H
+#define HOP_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hop_ctx hop_ctx;
+typedef struct hop_trace hop_trace;
+
+typedef enum hop_status {
+    HOP_OK = 0,
+    HOP_E_ARG = -1,         /* null pointer, negative size, unknown option ...                    */
+    HOP_E_GRAPH = -2,       /* missing self-loop, duplicate edge, b >= |N_in(i)|, max_skip > s+1  */
+    HOP_E_TRACE = -3,       /* trace record violates the protocol (see hop_load_trace)            */
+    HOP_E_STATE = -4,       /* call out of order: no buffers bound, no trace loaded, past the end */
+    HOP_E_DEADLOCK = -5,    /* the simulated protocol cannot make progress                        */
+    HOP_E_CUDA = -6,        /* a CUDA runtime call failed (message has the CUDA error string)     */
+    HOP_E_DEVICE = -7,      /* a kernel reported a failed internal check (see hop_read_status)    */
+    HOP_E_UNSUPPORTED = -8  /* combination not implemented (e.g. momentum with the CSR SVM mode)  */
+} hop_status;
+
+/* Per (level, worker) operation in a trace. */
+typedef enum hop_op {
+    HOP_OP_IDLE = 0,    /* the worker skipped this iteration (Section 5)                          */
+    HOP_OP_NORMAL = 1,  /* Compute + Recv + Reduce + Apply of Fig. alg2                           */
+    HOP_OP_JUMP = 2     /* Recv(k) + Reduce of the worker's current parameters before a jump to   */
+                        /* iteration k+1 (Section 5); no gradient                                  */
+} hop_op;
+
+/* Reduce weights. UNIFORM: 1/|consumed| (Fig. alg4 Reduce; Eq. 1 when everything is consumed).
+ * STALE_LINEAR: numerator Iter(u) - (k - s) + 1, normalised (Eq. 2). */
+typedef enum hop_weight_mode { HOP_W_UNIFORM = 0, HOP_W_STALE_LINEAR = 1 } hop_weight_mode;
+
+/* Where the gradient of a level comes from. */
+typedef enum hop_grad_mode {
+    HOP_GRAD_EXTERNAL = 0,   /* the caller fills G before each hop_step                            */
+    HOP_GRAD_SYNTHETIC = 1,  /* G[i][p] = sigma * normal(seed, i, k, p): Philox4x32-10 with counter */
+                             /* (p/4, i, k, 6), key = seed, Box-Muller on 23-bit uniforms          */
+    HOP_GRAD_SVM_DENSE = 2,  /* hinge-loss linear SVM, dense rows (hop_bind_svm_dense)             */
+    HOP_GRAD_SVM_CSR = 3     /* hinge-loss linear SVM, CSR rows (hop_bind_svm_csr)                 */
+} hop_grad_mode;
+
+typedef enum hop_mix_kernel {
+    HOP_MIX_AUTO = 0,
+    HOP_MIX_STAGED = 1,      /* column tile staged in shared memory with ordinary vector loads     */
+    HOP_MIX_BULK = 2,        /* same, slices fetched by asynchronous bulk copies in a pipeline     */
+    HOP_MIX_TENSOR = 3       /* dense graphs: W_k * X on tcgen05 tensor cores, 3xTF32              */
+} hop_mix_kernel;
+
+typedef enum hop_option {
+    HOP_OPT_MAX_IG = 1,       /* token-queue bound max_ig >= 1 (Section 4.2); 0 = no token queues;  */
+                              /* default max(1, s)                                                  */
+    HOP_OPT_LR = 2,           /* learning rate eta (default 0.1)                                    */
+    HOP_OPT_MOMENTUM = 3,     /* mu; m <- mu*m + g, x <- mix - eta*m; buffers local (default 0)     */
+    HOP_OPT_WEIGHT_MODE = 4,  /* hop_weight_mode (default UNIFORM)                                  */
+    HOP_OPT_GRAD_MODE = 5,    /* hop_grad_mode (default EXTERNAL)                                   */
+    HOP_OPT_GRAD_SEED = 6,    /* integer < 2^53                                                     */
+    HOP_OPT_GRAD_SIGMA = 7,   /* default 1e-3                                                       */
+    HOP_OPT_MIX_KERNEL = 8,   /* hop_mix_kernel (default AUTO)                                      */
+    HOP_OPT_COL_OFFSET = 9,   /* global index of local parameter 0 when P is a shard of a larger    */
+                              /* vector (multiple of 4); only the synthetic gradient reads it       */
+    HOP_OPT_BACKUP_OF_WORKER = 1000 /* key = 1000 + i sets N_buw(i) of one worker (Fig. alg4)       */
+} hop_option;
+
+/* ---- context -------------------------------------------------------------------------------
+ * Problem statement of Figs. alg1-alg4: graph G (in-neighbour lists in CSR form, self-loop
+ * required at every node, Section 3.1), N workers, P parameters, staleness bound s >= 0
+ * (max_staleness of Fig. alg3), backup workers b (N_buw, the same for every worker; must be
+ * < |N_in(i)|), max_skip >= 0 = largest number of iterations skipped in one jump (0 disables
+ * skipping; <= s+1 so that the jumper's parameters are still inside its version ring).
+ * in_ptr[N+1] and in_idx[in_ptr[N]] are host arrays, copied.  Touches no GPU. */
+int hop_create(hop_ctx** out, const int32_t* in_ptr, const int32_t* in_idx,
+               int32_t N, int64_t P, int32_t s, int32_t b, int32_t max_skip);
+int hop_destroy(hop_ctx* ctx);
+const char* hop_last_error(const hop_ctx* ctx);
+int hop_set_option(hop_ctx* ctx, int key, double value);
+
+/* ---- protocol simulation (host only, no GPU) --------------------------------------------------
+ * ticks[N][iters] (host): Compute of worker i in iteration k lasts ticks[i*iters+k] >= 1 time
+ * units; every other operation is instantaneous.  Runs Train() of Fig. alg2 for all workers with
+ * Recv of Figs. alg3/alg4 and the skipping rule of Section 5 and returns the consumption trace.
+ * HOP_E_DEADLOCK if no worker can move before all are finished. */
+int hop_sim_run(hop_ctx* ctx, const uint64_t* ticks, int32_t iters, hop_trace** out);
+
+/* A trace from caller-supplied host arrays (copied): op[levels*N]; ptr[levels*N+1] offsets into
+ * nbr/ver/num (record of (k,i) = [ptr[k*N+i], ptr[k*N+i+1])); den[levels*N]. */
+int hop_trace_create(hop_trace** out, int32_t levels, int32_t N, const int32_t* op,
+                     const int64_t* ptr, const int32_t* nbr, const int32_t* ver,
+                     const int32_t* num, const int32_t* den);
+int hop_trace_dims(const hop_trace* t, int32_t* levels, int32_t* N, int64_t* entries,
+                   uint64_t* makespan_ticks);
+/* Copies the trace into caller arrays of the sizes given by hop_trace_dims (any may be NULL). */
+int hop_trace_export(const hop_trace* t, int32_t* op, int64_t* ptr, int32_t* nbr, int32_t* ver,
+                     int32_t* num, int32_t* den);
+int hop_trace_destroy(hop_trace* t);
+
+/* ---- device buffers ---------------------------------------------------------------------------
+ * X, M, G: device pointers laid out as above, 16-byte aligned; M may be NULL when momentum is 0,
+ * G may be NULL in CSR SVM mode.  cuda_stream is a cudaStream_t (NULL = default stream). */
+int hop_bind_buffers(hop_ctx* ctx, float* X, float* M, float* G, void* cuda_stream);
+
+/* Hinge-loss linear SVM without bias or regulariser: margin_r = a_r . x_{k,i};
+ * coef_r = -y_r / batch if y_r * margin_r < 1 else 0; g = sum_r coef_r a_r.  The minibatch of
+ * iteration k is rows [(k mod (rows_per_worker/batch)) * batch, +batch) of the worker's shard.
+ * Dense: A[N][rows_per_worker][P], y[N][rows_per_worker] (device).  CSR: row_ptr[N*rows+1]
+ * (global offsets), col, val, y (device).  Allocates N*batch floats of device scratch. */
+int hop_bind_svm_dense(hop_ctx* ctx, const float* A, const float* y,
+                       int32_t rows_per_worker, int32_t batch);
+int hop_bind_svm_csr(hop_ctx* ctx, const int64_t* row_ptr, const int32_t* col, const float* val,
+                     const float* y, int32_t rows_per_worker, int32_t batch);
+
+/* Validates every record on the host -- consumed neighbour in N_in(i), version in [k-s, k] and
+ * actually produced, own update present, at least |N_in(i)| - b entries, positive numerators
+ * summing to den, JUMP/IDLE consistent with the versions a worker holds -- then uploads the
+ * per-level tables (cudaMalloc + H2D on the bound stream) and rewinds to level 0. */
+int hop_load_trace(hop_ctx* ctx, const hop_trace* t);
+
+/* Version `version` of worker `worker` (-1 = every worker) <- host_src[P]; synchronous. */
+int hop_write_params(hop_ctx* ctx, int32_t worker, int32_t version, const float* host_src);
+/* host_dst[P] <- version `version` (-1 = newest the worker holds after the executed levels) of
+ * worker `worker`; synchronises the stream. */
+int hop_read_params(hop_ctx* ctx, int32_t worker, int32_t version, float* host_dst);
+/* Newest version worker holds after the levels executed so far. */
+int hop_newest_version(hop_ctx* ctx, int32_t worker, int32_t* version);
+
+/* Next level to execute (momentum buffers are not touched). */
+int hop_set_level(hop_ctx* ctx, int32_t level);
+/* Executes the next level k of the loaded trace for all N workers: gradient kernels on slot k,
+ * then the fused gather-mix-update writing slot k+1, then (CSR SVM) the sparse apply.
+ * Asynchronous; HOP_E_STATE past the end of the trace. */
+int hop_step(hop_ctx* ctx);
+/* Same for one level handed in from the host (streaming use: the protocol decides level by
+ * level): validates the records, uploads them from a pinned staging buffer, executes the level,
+ * copies the first probe_len floats of worker 0's new version into probe_dst (host, may be NULL)
+ * and synchronises.  op[N], ptr[N+1], den[N]; nbr/ver/num as in hop_trace_create. */
+int hop_step_host(hop_ctx* ctx, const int32_t* op, const int64_t* ptr, const int32_t* nbr,
+                  const int32_t* ver, const int32_t* num, const int32_t* den,
+                  float* probe_dst, int64_t probe_len);
+
+/* Synchronises and returns the device-side error word (0 = no kernel check failed; otherwise
+ * a code in the top byte and a detail in the rest). */
+int hop_read_status(hop_ctx* ctx, int32_t* device_error_word);
+
+/* out[8] (host) for a level of the loaded trace: distinct consumed slices U_k, NORMAL records,
+ * JUMP records, consumed entries sum_i |C_{i,k}|, tile width chosen, kernel chosen, staged rows,
+ * algorithmic bytes of the mix-update kernel. */
+int hop_level_stats(hop_ctx* ctx, int32_t level, int64_t* out);
+/* Number of kernels launched by this context so far. */
+int hop_launch_count(hop_ctx* ctx, int64_t* launches);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HOP_B200_H */

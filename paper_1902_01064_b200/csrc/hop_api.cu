@@ -1,0 +1,476 @@
+// C ABI of libhop_b200.so: context, options, buffer binding, trace upload, level execution.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "hop_internal.h"
+
+const char* hop_trace_last_error();
+
+struct hop_ctx {
+    HopGraph g;
+    HopSimParams sp;
+    int64_t P = 0;
+    int32_t s = 0;
+    // options
+    double lr = 0.1, momentum = 0.0, sigma = 1e-3;
+    int32_t grad_mode = HOP_GRAD_EXTERNAL, mix_kernel = HOP_MIX_AUTO;
+    uint64_t grad_seed = 0;
+    int64_t col_offset = 0;
+    // bound device memory (borrowed)
+    float *X = nullptr, *M = nullptr, *G = nullptr;
+    cudaStream_t stream = nullptr;
+    bool bound = false;
+    // SVM data (borrowed) + coefficient scratch (owned)
+    const float *svmA = nullptr, *svmY = nullptr, *svmVal = nullptr;
+    const int64_t* svmRowPtr = nullptr;
+    const int32_t* svmCol = nullptr;
+    int32_t svmR = 0, svmB = 0;
+    float* coef = nullptr;
+    // loaded trace (owned device tables)
+    std::vector<HopLevelHost> levels;
+    int32_t* d_i32 = nullptr;       // src_row and grad_workers of all levels
+    HopRecord* d_rec = nullptr;
+    HopEntry* d_ent = nullptr;
+    bool loaded = false;
+    // streaming mode (hop_step_host): pinned staging + device copy of one level
+    void* h_stage = nullptr; void* d_stage = nullptr; size_t stage_cap = 0;
+    float* h_probe = nullptr; size_t probe_cap = 0;
+    // progress
+    int32_t level = 0;
+    std::vector<int32_t> newest;
+    std::vector<std::vector<uint8_t>> sent;   // [N][level] worker entered (sent) that iteration
+    int32_t* d_err = nullptr;
+    int sm_count = 0;
+    int64_t launches = 0;
+    std::string err;
+};
+
+static std::string g_create_err;
+
+#define HOP_FAIL(ctx, code, msg) do { (ctx)->err = (msg); return (code); } while (0)
+#define HOP_CUDA(ctx, call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { \
+    (ctx)->err = std::string(#call) + ": " + cudaGetErrorString(e_); return HOP_E_CUDA; } } while (0)
+
+extern "C" const char* hop_last_error(const hop_ctx* ctx) {
+    if (ctx) return ctx->err.c_str();
+    const char* t = hop_trace_last_error();
+    return g_create_err.empty() ? t : g_create_err.c_str();
+}
+
+extern "C" int hop_create(hop_ctx** out, const int32_t* in_ptr, const int32_t* in_idx, int32_t N, int64_t P,
+                          int32_t s, int32_t b, int32_t max_skip) {
+    g_create_err.clear();
+    auto fail = [&](int code, const std::string& m) { g_create_err = "hop_create: " + m; return code; };
+    if (!out || !in_ptr || !in_idx) return fail(HOP_E_ARG, "null pointer");
+    if (N <= 0 || P <= 0 || s < 0 || b < 0 || max_skip < 0) return fail(HOP_E_ARG, "N, P must be positive; s, b, max_skip non-negative");
+    if ((int64_t)N * (s + 1) > (1 << 30)) return fail(HOP_E_ARG, "N*(s+1) too large");
+    if (max_skip > s + 1) return fail(HOP_E_GRAPH, "max_skip > s+1: the jumper's parameters would leave its version ring");
+    if (in_ptr[0] != 0) return fail(HOP_E_GRAPH, "in_ptr[0] != 0");
+    hop_ctx* c = new hop_ctx;
+    c->g.N = N;
+    c->g.in_ptr.assign(in_ptr, in_ptr + N + 1);
+    std::vector<std::vector<int32_t>> outs(N);
+    for (int32_t i = 0; i < N; ++i) {
+        if (in_ptr[i + 1] < in_ptr[i]) { delete c; return fail(HOP_E_GRAPH, "in_ptr not monotone"); }
+        std::vector<int32_t> nb(in_idx + in_ptr[i], in_idx + in_ptr[i + 1]);
+        std::sort(nb.begin(), nb.end());
+        if (std::adjacent_find(nb.begin(), nb.end()) != nb.end()) { delete c; return fail(HOP_E_GRAPH, "duplicate in-neighbour at worker " + std::to_string(i)); }
+        if (!nb.empty() && (nb.front() < 0 || nb.back() >= N)) { delete c; return fail(HOP_E_GRAPH, "neighbour id out of range at worker " + std::to_string(i)); }
+        if (!std::binary_search(nb.begin(), nb.end(), i)) { delete c; return fail(HOP_E_GRAPH, "worker " + std::to_string(i) + " has no self-loop"); }
+        if (b >= (int32_t)nb.size()) { delete c; return fail(HOP_E_GRAPH, "b >= |N_in(" + std::to_string(i) + ")|"); }
+        for (int32_t j : nb) outs[j].push_back(i);
+        c->g.in_idx.insert(c->g.in_idx.end(), nb.begin(), nb.end());
+    }
+    c->g.out_ptr.assign(1, 0);
+    for (int32_t j = 0; j < N; ++j) {
+        c->g.out_idx.insert(c->g.out_idx.end(), outs[j].begin(), outs[j].end());
+        c->g.out_ptr.push_back((int32_t)c->g.out_idx.size());
+    }
+    c->P = P; c->s = s;
+    c->sp.s = s; c->sp.max_ig = std::max(1, s); c->sp.max_skip = max_skip; c->sp.weight_mode = HOP_W_UNIFORM;
+    c->sp.b.assign(N, b);
+    c->newest.assign(N, 0);
+    c->sent.assign(N, {});
+    *out = c;
+    return HOP_OK;
+}
+
+static void free_trace_tables(hop_ctx* c) {
+    if (c->d_i32) cudaFree(c->d_i32);
+    if (c->d_rec) cudaFree(c->d_rec);
+    if (c->d_ent) cudaFree(c->d_ent);
+    c->d_i32 = nullptr; c->d_rec = nullptr; c->d_ent = nullptr;
+    c->levels.clear();
+    c->loaded = false;
+}
+
+extern "C" int hop_destroy(hop_ctx* c) {
+    if (!c) return HOP_OK;
+    free_trace_tables(c);
+    if (c->coef) cudaFree(c->coef);
+    if (c->d_err) cudaFree(c->d_err);
+    if (c->d_stage) cudaFree(c->d_stage);
+    if (c->h_stage) cudaFreeHost(c->h_stage);
+    if (c->h_probe) cudaFreeHost(c->h_probe);
+    delete c;
+    return HOP_OK;
+}
+
+extern "C" int hop_set_option(hop_ctx* c, int key, double v) {
+    if (!c) return HOP_E_ARG;
+    if (key >= HOP_OPT_BACKUP_OF_WORKER) {
+        const int i = key - HOP_OPT_BACKUP_OF_WORKER;
+        if (i >= c->g.N) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: worker index out of range");
+        const int d = c->g.in_ptr[i + 1] - c->g.in_ptr[i];
+        if (v < 0 || v >= d || v != std::floor(v)) HOP_FAIL(c, HOP_E_GRAPH, "hop_set_option: N_buw(i) must be an integer in [0, |N_in(i)|)");
+        c->sp.b[i] = (int32_t)v;
+        return HOP_OK;
+    }
+    switch (key) {
+    case HOP_OPT_MAX_IG:
+        if (v < 0 || v != std::floor(v)) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: max_ig must be a non-negative integer");
+        c->sp.max_ig = (int32_t)v; break;
+    case HOP_OPT_LR: c->lr = v; break;
+    case HOP_OPT_MOMENTUM: c->momentum = v; break;
+    case HOP_OPT_WEIGHT_MODE:
+        if (v != HOP_W_UNIFORM && v != HOP_W_STALE_LINEAR) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: unknown weight mode");
+        c->sp.weight_mode = (int32_t)v; break;
+    case HOP_OPT_GRAD_MODE:
+        if (v < 0 || v > 3 || v != std::floor(v)) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: unknown gradient mode");
+        c->grad_mode = (int32_t)v; break;
+    case HOP_OPT_GRAD_SEED:
+        if (v < 0 || v >= 9007199254740992.0 || v != std::floor(v)) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: seed must be an integer in [0, 2^53)");
+        c->grad_seed = (uint64_t)v; break;
+    case HOP_OPT_GRAD_SIGMA: c->sigma = v; break;
+    case HOP_OPT_MIX_KERNEL:
+        if (v < 0 || v > 3 || v != std::floor(v)) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: unknown mix kernel");
+        c->mix_kernel = (int32_t)v; break;
+    case HOP_OPT_COL_OFFSET:
+        if (v < 0 || v != std::floor(v) || std::fmod(v, 4.0) != 0.0) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: column offset must be a non-negative multiple of 4");
+        c->col_offset = (int64_t)v; break;
+    default: HOP_FAIL(c, HOP_E_ARG, "hop_set_option: unknown key " + std::to_string(key));
+    }
+    return HOP_OK;
+}
+
+extern "C" int hop_sim_run(hop_ctx* c, const uint64_t* ticks, int32_t iters, hop_trace** out) {
+    if (!c || !ticks || !out || iters <= 0) { if (c) c->err = "hop_sim_run: bad argument"; return HOP_E_ARG; }
+    hop_trace* t = new hop_trace;
+    const int rc = hop_simulate(c->g, c->sp, ticks, iters, *t, c->err);
+    if (rc != HOP_OK) { delete t; return rc; }
+    *out = t;
+    return HOP_OK;
+}
+
+// ---- device ------------------------------------------------------------------------------------
+static int ensure_device(hop_ctx* c) {
+    if (c->d_err) return HOP_OK;
+    int dev = 0;
+    HOP_CUDA(c, cudaGetDevice(&dev));
+    HOP_CUDA(c, cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev));
+    HOP_CUDA(c, cudaMalloc(&c->d_err, sizeof(int32_t)));
+    HOP_CUDA(c, cudaMemset(c->d_err, 0, sizeof(int32_t)));
+    return HOP_OK;
+}
+
+extern "C" int hop_bind_buffers(hop_ctx* c, float* X, float* M, float* G, void* stream) {
+    if (!c) return HOP_E_ARG;
+    if (!X) HOP_FAIL(c, HOP_E_ARG, "hop_bind_buffers: X is null");
+    if (((uintptr_t)X | (uintptr_t)M | (uintptr_t)G) & 15) HOP_FAIL(c, HOP_E_ARG, "hop_bind_buffers: pointers must be 16-byte aligned");
+    const int rc = ensure_device(c);
+    if (rc) return rc;
+    c->X = X; c->M = M; c->G = G; c->stream = (cudaStream_t)stream; c->bound = true;
+    return HOP_OK;
+}
+
+static int alloc_coef(hop_ctx* c, int32_t R, int32_t B) {
+    if (R <= 0 || B <= 0 || R % B != 0) HOP_FAIL(c, HOP_E_ARG, "SVM shard: rows_per_worker must be a positive multiple of batch");
+    const int rc = ensure_device(c);
+    if (rc) return rc;
+    if (c->coef) { cudaFree(c->coef); c->coef = nullptr; }
+    HOP_CUDA(c, cudaMalloc(&c->coef, (size_t)c->g.N * B * sizeof(float)));
+    c->svmR = R; c->svmB = B;
+    return HOP_OK;
+}
+
+extern "C" int hop_bind_svm_dense(hop_ctx* c, const float* A, const float* y, int32_t R, int32_t B) {
+    if (!c) return HOP_E_ARG;
+    if (!A || !y) HOP_FAIL(c, HOP_E_ARG, "hop_bind_svm_dense: null pointer");
+    const int rc = alloc_coef(c, R, B);
+    if (rc) return rc;
+    c->svmA = A; c->svmY = y;
+    return HOP_OK;
+}
+
+extern "C" int hop_bind_svm_csr(hop_ctx* c, const int64_t* row_ptr, const int32_t* col, const float* val,
+                                const float* y, int32_t R, int32_t B) {
+    if (!c) return HOP_E_ARG;
+    if (!row_ptr || !col || !val || !y) HOP_FAIL(c, HOP_E_ARG, "hop_bind_svm_csr: null pointer");
+    const int rc = alloc_coef(c, R, B);
+    if (rc) return rc;
+    c->svmRowPtr = row_ptr; c->svmCol = col; c->svmVal = val; c->svmY = y;
+    return HOP_OK;
+}
+
+// Tile width and kernel for one level: as many columns per tile as the staged rows leave room for.
+static int plan_level(hop_ctx* c, HopLevelHost& L) {
+    const bool use_g = c->grad_mode != HOP_GRAD_SVM_CSR;
+    const bool mom = c->momentum != 0.0;
+    const int nG = use_g ? L.nG : 0;
+    L.stage_rows = L.U + nG * (mom ? 2 : 1);
+    int kernel = c->mix_kernel;
+    if (kernel == HOP_MIX_AUTO || kernel == HOP_MIX_TENSOR) kernel = (c->P % 4 == 0) ? HOP_MIX_BULK : HOP_MIX_STAGED;
+    if (kernel == HOP_MIX_BULK && c->P % 4 != 0) HOP_FAIL(c, HOP_E_UNSUPPORTED, "the bulk-copy mix kernel needs P to be a multiple of 4");
+    const int rows = std::max(1, L.stage_rows);
+    const int64_t budget = hop_mix_smem_budget(kernel) / hop_mix_stages(kernel);
+    int64_t w = budget / ((int64_t)rows * 4);
+    const int unit = (c->P % 4 == 0) ? 4 : 1;
+    if (w >= 128) w = std::min<int64_t>(1024, w / 128 * 128);
+    else if (w >= 32) w = w / 32 * 32;
+    else w = w / unit * unit;
+    if (w < unit) HOP_FAIL(c, HOP_E_UNSUPPORTED, "a level consumes more distinct slices than shared memory can stage");
+    const int64_t Pr = (c->P + unit - 1) / unit * unit;
+    w = std::min<int64_t>(w, Pr);
+    L.tile_w = (int32_t)w;
+    L.kernel = kernel;
+    // every distinct consumed slice once + gradient once + result once (+ momentum read and write)
+    L.alg_bytes = 4 * c->P * ((int64_t)L.U + nG + L.nA + (mom ? 2 * (int64_t)nG : 0));
+    return HOP_OK;
+}
+
+extern "C" int hop_load_trace(hop_ctx* c, const hop_trace* t) {
+    if (!c || !t) return HOP_E_ARG;
+    if (!c->bound) HOP_FAIL(c, HOP_E_STATE, "hop_load_trace: bind buffers first");
+    if (t->N != c->g.N) HOP_FAIL(c, HOP_E_TRACE, "hop_load_trace: trace has a different number of workers");
+    const int32_t N = t->N, L = t->levels;
+    std::vector<int32_t> newest(N, 0);
+    std::vector<std::vector<uint8_t>> sent(N, std::vector<uint8_t>(L, 0));
+    for (int32_t k = 0; k < L; ++k)
+        for (int32_t i = 0; i < N; ++i) sent[i][k] = t->op[(size_t)k * N + i] == HOP_OP_NORMAL;
+    std::vector<HopLevelHost> levels(L);
+    for (int32_t k = 0; k < L; ++k) {
+        const size_t r = (size_t)k * N;
+        const int rc = hop_validate_level(c->g, c->sp, k, &t->op[r], &t->ptr[r], t->nbr.data(), t->ver.data(),
+                                          t->num.data(), &t->den[r], newest, &sent, c->err);
+        if (rc) return rc;
+        hop_build_level(c->g, c->s, k, &t->op[r], &t->ptr[r], t->nbr.data(), t->ver.data(), t->num.data(), &t->den[r], levels[k]);
+        const int rc2 = plan_level(c, levels[k]);
+        if (rc2) return rc2;
+    }
+    std::vector<int32_t> h_i32; std::vector<HopRecord> h_rec; std::vector<HopEntry> h_ent;
+    for (auto& Lv : levels) {
+        Lv.off_src = (int64_t)h_i32.size(); h_i32.insert(h_i32.end(), Lv.src_row.begin(), Lv.src_row.end());
+        Lv.off_gw = (int64_t)h_i32.size(); h_i32.insert(h_i32.end(), Lv.grad_workers.begin(), Lv.grad_workers.end());
+        Lv.off_rec = (int64_t)h_rec.size(); h_rec.insert(h_rec.end(), Lv.recs.begin(), Lv.recs.end());
+        Lv.off_ent = (int64_t)h_ent.size(); h_ent.insert(h_ent.end(), Lv.ents.begin(), Lv.ents.end());
+    }
+    free_trace_tables(c);
+    HOP_CUDA(c, cudaMalloc(&c->d_i32, std::max<size_t>(1, h_i32.size()) * sizeof(int32_t)));
+    HOP_CUDA(c, cudaMalloc(&c->d_rec, std::max<size_t>(1, h_rec.size()) * sizeof(HopRecord)));
+    HOP_CUDA(c, cudaMalloc(&c->d_ent, std::max<size_t>(1, h_ent.size()) * sizeof(HopEntry)));
+    HOP_CUDA(c, cudaMemcpyAsync(c->d_i32, h_i32.data(), h_i32.size() * sizeof(int32_t), cudaMemcpyHostToDevice, c->stream));
+    HOP_CUDA(c, cudaMemcpyAsync(c->d_rec, h_rec.data(), h_rec.size() * sizeof(HopRecord), cudaMemcpyHostToDevice, c->stream));
+    HOP_CUDA(c, cudaMemcpyAsync(c->d_ent, h_ent.data(), h_ent.size() * sizeof(HopEntry), cudaMemcpyHostToDevice, c->stream));
+    HOP_CUDA(c, cudaStreamSynchronize(c->stream));   // the host vectors go out of scope
+    c->levels = std::move(levels);
+    c->sent = std::move(sent);
+    c->loaded = true;
+    c->level = 0;
+    std::fill(c->newest.begin(), c->newest.end(), 0);
+    return HOP_OK;
+}
+
+static int check_mode(hop_ctx* c) {
+    const bool mom = c->momentum != 0.0;
+    if (mom && !c->M) HOP_FAIL(c, HOP_E_STATE, "momentum != 0 but no momentum buffer bound");
+    if (c->grad_mode != HOP_GRAD_SVM_CSR && !c->G) HOP_FAIL(c, HOP_E_STATE, "this gradient mode needs a dense gradient buffer G");
+    if (c->grad_mode == HOP_GRAD_SVM_CSR && mom) HOP_FAIL(c, HOP_E_UNSUPPORTED, "momentum with the CSR SVM mode is not implemented");
+    if (c->grad_mode == HOP_GRAD_SVM_CSR && !c->svmRowPtr) HOP_FAIL(c, HOP_E_STATE, "CSR SVM mode without hop_bind_svm_csr");
+    if (c->grad_mode == HOP_GRAD_SVM_DENSE && !c->svmA) HOP_FAIL(c, HOP_E_STATE, "dense SVM mode without hop_bind_svm_dense");
+    return HOP_OK;
+}
+
+// Enqueues the kernels of one level.
+static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv) {
+    HopLaunchCfg cfg{};
+    cfg.X = c->X; cfg.M = c->M; cfg.G = c->G; cfg.P = c->P; cfg.N = c->g.N; cfg.s = c->s;
+    cfg.lr = (float)c->lr; cfg.mu = (float)c->momentum; cfg.tile_w = L.tile_w;
+    cfg.use_g = c->grad_mode != HOP_GRAD_SVM_CSR;
+    cfg.sm_count = c->sm_count; cfg.err_word = c->d_err; cfg.stream = c->stream;
+    int e = 0;
+    if (L.nG > 0) {
+        switch (c->grad_mode) {
+        case HOP_GRAD_SYNTHETIC:
+            e = hop_launch_synth_grad(cfg, lv, c->grad_seed, (float)c->sigma, c->col_offset); c->launches += 1; break;
+        case HOP_GRAD_SVM_DENSE:
+            e = hop_launch_svm_dense(cfg, lv, c->svmA, c->svmY, c->svmR, c->svmB, c->coef); c->launches += 2; break;
+        case HOP_GRAD_SVM_CSR:
+            e = hop_launch_svm_csr_coef(cfg, lv, c->svmRowPtr, c->svmCol, c->svmVal, c->svmY, c->svmR, c->svmB, c->coef); c->launches += 1; break;
+        default: break;
+        }
+        if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("gradient kernel launch: ") + cudaGetErrorString((cudaError_t)e));
+    }
+    if (L.nA > 0) {
+        e = (L.kernel == HOP_MIX_BULK) ? hop_launch_mix_bulk(cfg, lv) : hop_launch_mix_staged(cfg, lv);
+        c->launches += 1;
+        if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("mix kernel launch: ") + cudaGetErrorString((cudaError_t)e));
+    }
+    if (L.nG > 0 && c->grad_mode == HOP_GRAD_SVM_CSR) {
+        e = hop_launch_svm_csr_apply(cfg, lv, c->svmRowPtr, c->svmCol, c->svmVal, c->svmR, c->svmB, c->coef);
+        c->launches += 1;
+        if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("sparse apply launch: ") + cudaGetErrorString((cudaError_t)e));
+    }
+    return HOP_OK;
+}
+
+extern "C" int hop_step(hop_ctx* c) {
+    if (!c) return HOP_E_ARG;
+    if (!c->bound || !c->loaded) HOP_FAIL(c, HOP_E_STATE, "hop_step: bind buffers and load a trace first");
+    if (c->level >= (int32_t)c->levels.size()) HOP_FAIL(c, HOP_E_STATE, "hop_step: past the end of the trace");
+    int rc = check_mode(c);
+    if (rc) return rc;
+    const HopLevelHost& L = c->levels[c->level];
+    HopLevelDev lv{c->d_i32 + L.off_src, c->d_rec + L.off_rec, c->d_ent + L.off_ent, c->d_i32 + L.off_gw,
+                   L.U, L.nA, L.nG, c->level};
+    rc = run_level(c, L, lv);
+    if (rc) return rc;
+    for (const HopRecord& r : L.recs) c->newest[r.worker] = c->level + 1;
+    c->level += 1;
+    return HOP_OK;
+}
+
+extern "C" int hop_step_host(hop_ctx* c, const int32_t* op, const int64_t* ptr, const int32_t* nbr, const int32_t* ver,
+                             const int32_t* num, const int32_t* den, float* probe_dst, int64_t probe_len) {
+    if (!c) return HOP_E_ARG;
+    if (!op || !ptr || !den) HOP_FAIL(c, HOP_E_ARG, "hop_step_host: null pointer");
+    if (!c->bound) HOP_FAIL(c, HOP_E_STATE, "hop_step_host: bind buffers first");
+    if (probe_len < 0 || probe_len > c->P) HOP_FAIL(c, HOP_E_ARG, "hop_step_host: probe_len out of range");
+    int rc = check_mode(c);
+    if (rc) return rc;
+    const int32_t N = c->g.N, k = c->level;
+    if (ptr[0] != 0) HOP_FAIL(c, HOP_E_ARG, "hop_step_host: ptr[0] must be 0");
+    for (int32_t i = 0; i < N; ++i) {
+        if ((int32_t)c->sent[i].size() <= k) c->sent[i].resize(k + 1, 0);
+        c->sent[i][k] = op[i] == HOP_OP_NORMAL;
+    }
+    std::vector<int32_t> newest = c->newest;
+    rc = hop_validate_level(c->g, c->sp, k, op, ptr, nbr, ver, num, den, newest, &c->sent, c->err);
+    if (rc) return rc;
+    HopLevelHost L;
+    hop_build_level(c->g, c->s, k, op, ptr, nbr, ver, num, den, L);
+    rc = plan_level(c, L);
+    if (rc) return rc;
+    // pack [src_row | grad_workers | recs | ents] into one pinned buffer, one H2D copy
+    const size_t b_src = L.src_row.size() * 4, b_gw = L.grad_workers.size() * 4;
+    const size_t o_gw = b_src, o_rec = (o_gw + b_gw + 15) / 16 * 16, b_rec = L.recs.size() * sizeof(HopRecord);
+    const size_t o_ent = o_rec + b_rec, b_ent = L.ents.size() * sizeof(HopEntry), total = std::max<size_t>(16, o_ent + b_ent);
+    if (total > c->stage_cap) {
+        if (c->d_stage) cudaFree(c->d_stage);
+        if (c->h_stage) cudaFreeHost(c->h_stage);
+        c->d_stage = nullptr; c->h_stage = nullptr; c->stage_cap = 0;
+        const size_t cap = std::max<size_t>(total * 2, 1 << 16);
+        HOP_CUDA(c, cudaMalloc(&c->d_stage, cap));
+        HOP_CUDA(c, cudaMallocHost(&c->h_stage, cap));
+        c->stage_cap = cap;
+    }
+    if ((size_t)probe_len > c->probe_cap) {
+        if (c->h_probe) cudaFreeHost(c->h_probe);
+        c->h_probe = nullptr; c->probe_cap = 0;
+        HOP_CUDA(c, cudaMallocHost((void**)&c->h_probe, (size_t)probe_len * sizeof(float)));
+        c->probe_cap = (size_t)probe_len;
+    }
+    unsigned char* h = (unsigned char*)c->h_stage;
+    if (b_src) std::memcpy(h, L.src_row.data(), b_src);
+    if (b_gw) std::memcpy(h + o_gw, L.grad_workers.data(), b_gw);
+    if (b_rec) std::memcpy(h + o_rec, L.recs.data(), b_rec);
+    if (b_ent) std::memcpy(h + o_ent, L.ents.data(), b_ent);
+    HOP_CUDA(c, cudaMemcpyAsync(c->d_stage, h, total, cudaMemcpyHostToDevice, c->stream));
+    unsigned char* d = (unsigned char*)c->d_stage;
+    HopLevelDev lv{(const int32_t*)d, (const HopRecord*)(d + o_rec), (const HopEntry*)(d + o_ent), (const int32_t*)(d + o_gw),
+                   L.U, L.nA, L.nG, k};
+    rc = run_level(c, L, lv);
+    if (rc) return rc;
+    c->newest = newest;
+    c->level += 1;
+    if (probe_dst && probe_len > 0) {
+        const float* src = c->X + ((int64_t)0 * (c->s + 1) + c->newest[0] % (c->s + 1)) * c->P;
+        HOP_CUDA(c, cudaMemcpyAsync(c->h_probe, src, (size_t)probe_len * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+    }
+    HOP_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (probe_dst && probe_len > 0) std::memcpy(probe_dst, c->h_probe, (size_t)probe_len * sizeof(float));
+    return HOP_OK;
+}
+
+extern "C" int hop_set_level(hop_ctx* c, int32_t level) {
+    if (!c) return HOP_E_ARG;
+    if (level < 0 || (c->loaded && level > (int32_t)c->levels.size())) HOP_FAIL(c, HOP_E_ARG, "hop_set_level: out of range");
+    // newest version held by each worker after levels [0, level)
+    std::fill(c->newest.begin(), c->newest.end(), 0);
+    if (c->loaded)
+        for (int32_t k = 0; k < level; ++k)
+            for (const HopRecord& r : c->levels[k].recs) c->newest[r.worker] = k + 1;
+    c->level = level;
+    return HOP_OK;
+}
+
+extern "C" int hop_newest_version(hop_ctx* c, int32_t worker, int32_t* version) {
+    if (!c || !version) return HOP_E_ARG;
+    if (worker < 0 || worker >= c->g.N) HOP_FAIL(c, HOP_E_ARG, "hop_newest_version: worker out of range");
+    *version = c->newest[worker];
+    return HOP_OK;
+}
+
+extern "C" int hop_write_params(hop_ctx* c, int32_t worker, int32_t version, const float* src) {
+    if (!c) return HOP_E_ARG;
+    if (!src || version < 0 || worker < -1 || worker >= c->g.N) HOP_FAIL(c, HOP_E_ARG, "hop_write_params: bad argument");
+    if (!c->bound) HOP_FAIL(c, HOP_E_STATE, "hop_write_params: bind buffers first");
+    const int S = c->s + 1;
+    const int lo = worker < 0 ? 0 : worker, hi = worker < 0 ? c->g.N : worker + 1;
+    for (int i = lo; i < hi; ++i)
+        HOP_CUDA(c, cudaMemcpyAsync(c->X + ((int64_t)i * S + version % S) * c->P, src, (size_t)c->P * sizeof(float),
+                                    cudaMemcpyHostToDevice, c->stream));
+    HOP_CUDA(c, cudaStreamSynchronize(c->stream));
+    return HOP_OK;
+}
+
+extern "C" int hop_read_params(hop_ctx* c, int32_t worker, int32_t version, float* dst) {
+    if (!c) return HOP_E_ARG;
+    if (!dst || worker < 0 || worker >= c->g.N || version < -1) HOP_FAIL(c, HOP_E_ARG, "hop_read_params: bad argument");
+    if (!c->bound) HOP_FAIL(c, HOP_E_STATE, "hop_read_params: bind buffers first");
+    const int S = c->s + 1;
+    const int v = version < 0 ? c->newest[worker] : version;
+    HOP_CUDA(c, cudaMemcpyAsync(dst, c->X + ((int64_t)worker * S + v % S) * c->P, (size_t)c->P * sizeof(float),
+                                cudaMemcpyDeviceToHost, c->stream));
+    HOP_CUDA(c, cudaStreamSynchronize(c->stream));
+    return HOP_OK;
+}
+
+extern "C" int hop_read_status(hop_ctx* c, int32_t* word) {
+    if (!c || !word) return HOP_E_ARG;
+    *word = 0;
+    if (!c->d_err) return HOP_OK;
+    HOP_CUDA(c, cudaStreamSynchronize(c->stream));
+    HOP_CUDA(c, cudaMemcpy(word, c->d_err, sizeof(int32_t), cudaMemcpyDeviceToHost));
+    if (*word != 0) HOP_FAIL(c, HOP_E_DEVICE, "a kernel gave up waiting (status word " + std::to_string(*word) + ")");
+    return HOP_OK;
+}
+
+extern "C" int hop_level_stats(hop_ctx* c, int32_t level, int64_t* out) {
+    if (!c || !out) return HOP_E_ARG;
+    if (!c->loaded || level < 0 || level >= (int32_t)c->levels.size()) HOP_FAIL(c, HOP_E_ARG, "hop_level_stats: no such level");
+    const HopLevelHost& L = c->levels[level];
+    out[0] = L.U; out[1] = L.nG; out[2] = L.nJump; out[3] = L.sumC; out[4] = L.tile_w; out[5] = L.kernel;
+    out[6] = L.stage_rows; out[7] = L.alg_bytes;
+    return HOP_OK;
+}
+
+extern "C" int hop_launch_count(hop_ctx* c, int64_t* n) {
+    if (!c || !n) return HOP_E_ARG;
+    *n = c->launches;
+    return HOP_OK;
+}

@@ -1,0 +1,100 @@
+// Internal declarations shared by the translation units of libhop_b200.so.
+#pragma once
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "hop.h"
+
+struct hop_trace {
+    int32_t levels = 0, N = 0;
+    uint64_t makespan = 0;
+    std::vector<int32_t> op;    // [levels*N]
+    std::vector<int64_t> ptr;   // [levels*N+1]
+    std::vector<int32_t> nbr, ver, num;
+    std::vector<int32_t> den;   // [levels*N]
+};
+
+// ---- device-side tables of one level (built on the host, uploaded once) -------------------------
+struct HopRecord {          // one active (NORMAL or JUMP) worker of a level
+    int32_t worker;
+    int32_t out_row;        // row of X that receives x_{k+1,i}: worker*(s+1) + (k+1) mod (s+1)
+    int32_t ent_begin;      // first entry (relative to the level's entry array)
+    int32_t ent_count;
+    int32_t g_stage;        // index among the level's NORMAL workers, -1 for JUMP
+    int32_t cur_row;        // row of X holding x_{k,i} (gradient input); -1 for JUMP
+    int32_t pad0, pad1;
+};
+struct HopEntry {
+    int32_t u;              // index into the level's distinct-slice list
+    float w;                // float(num) / float(den)
+};
+
+struct HopLevelHost {
+    int32_t U = 0, nA = 0, nG = 0, nJump = 0;
+    int64_t sumC = 0;
+    std::vector<int32_t> src_row;       // [U] rows of X
+    std::vector<HopRecord> recs;        // [nA]
+    std::vector<HopEntry> ents;
+    std::vector<int32_t> grad_workers;  // [nG] workers with a NORMAL record
+    // offsets into the uploaded arrays
+    int64_t off_src = 0, off_rec = 0, off_ent = 0, off_gw = 0;
+    // launch plan
+    int32_t tile_w = 0, kernel = 0, stage_rows = 0;
+    int64_t alg_bytes = 0;
+};
+
+struct HopLevelDev {        // passed by value to the kernels
+    const int32_t* src_row;
+    const HopRecord* recs;
+    const HopEntry* ents;
+    const int32_t* grad_workers;
+    int32_t U, nA, nG, level;
+};
+
+struct HopGraph {
+    int32_t N = 0;
+    std::vector<int32_t> in_ptr, in_idx;    // in-neighbours, self included
+    std::vector<int32_t> out_ptr, out_idx;  // out-neighbours, self included
+};
+
+struct HopSimParams {
+    int32_t s, max_ig /*0 = none*/, max_skip, weight_mode;
+    std::vector<int32_t> b;
+};
+
+// hop_sim.cpp
+int hop_simulate(const HopGraph& g, const HopSimParams& p, const uint64_t* ticks, int32_t iters,
+                 hop_trace& out, std::string& err);
+// hop_trace.cpp
+int hop_validate_level(const HopGraph& g, const HopSimParams& p, int32_t level, const int32_t* op,
+                       const int64_t* ptr, const int32_t* nbr, const int32_t* ver, const int32_t* num,
+                       const int32_t* den, std::vector<int32_t>& newest,
+                       std::vector<std::vector<uint8_t>>* sent, std::string& err);
+void hop_build_level(const HopGraph& g, int32_t s, int32_t level, const int32_t* op, const int64_t* ptr,
+                     const int32_t* nbr, const int32_t* ver, const int32_t* num, const int32_t* den,
+                     HopLevelHost& out);
+
+// hop_kernels.cu : launchers.  All return a cudaError_t cast to int.
+struct HopLaunchCfg {
+    float* X; float* M; float* G;
+    int64_t P;
+    int32_t N, s;
+    float lr, mu;
+    int32_t tile_w;
+    int32_t use_g;      // dense gradient rows are applied
+    int32_t sm_count;
+    int32_t* err_word;  // device
+    void* stream;
+};
+int hop_launch_mix_staged(const HopLaunchCfg& c, const HopLevelDev& lv);
+int hop_launch_mix_bulk(const HopLaunchCfg& c, const HopLevelDev& lv);
+int hop_launch_synth_grad(const HopLaunchCfg& c, const HopLevelDev& lv, uint64_t seed, float sigma, int64_t col_offset);
+int hop_launch_svm_dense(const HopLaunchCfg& c, const HopLevelDev& lv, const float* A, const float* y,
+                         int32_t R, int32_t B, float* coef);
+int hop_launch_svm_csr_coef(const HopLaunchCfg& c, const HopLevelDev& lv, const int64_t* row_ptr, const int32_t* col,
+                            const float* val, const float* y, int32_t R, int32_t B, float* coef);
+int hop_launch_svm_csr_apply(const HopLaunchCfg& c, const HopLevelDev& lv, const int64_t* row_ptr, const int32_t* col,
+                             const float* val, int32_t R, int32_t B, const float* coef);
+int hop_mix_smem_budget(int kernel);   // usable dynamic shared memory per CTA for the kernel
+int hop_mix_stages(int kernel);

@@ -1,0 +1,429 @@
+// CUDA kernels of the Hop hot path for sm_100a.
+//
+//   mix_staged / mix_bulk   fused Recv-Reduce-Apply for one level: x_{k+1,i} = sum w * x_{v,j} - lr * d
+//                           (Fig. alg0 steps 2-3, Reduce of Fig. alg4 / Eq. 2), SGD or momentum
+//   synth_grad              G[i][p] = sigma * normal(seed, i, k, p)
+//   svm_margin_* / svm_dense_grad / svm_csr_apply   hinge-loss linear SVM gradient and sparse Apply
+//
+// In-place ring: version k+1 of a worker overwrites the slot of version k-s, which other workers may
+// consume in the same level.  A thread block therefore owns a column tile for ALL workers: it first
+// brings every distinct consumed slice of the tile into shared memory, then writes.  Blocks own
+// disjoint columns, so no other ordering is needed, and every distinct slice is read once.
+#include <cuda_runtime.h>
+#include <cstdint>
+
+#include "hop_internal.h"
+
+namespace {
+
+constexpr int kStagedThreads = 256;
+constexpr int kConsumerWarps = 8;
+constexpr int kBulkThreads = 32 * (kConsumerWarps + 1);
+constexpr int kBulkStages = 2;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+enum : int32_t { ERR_FULL_WAIT = 1 << 24, ERR_EMPTY_WAIT = 2 << 24 };
+
+// ------------------------------------------------------------------------------------------------
+// Consumer math shared by both mix kernels: one warp produces the tile of one record.
+// stage: [rows][w] floats; rows [0,U) consumed slices, [U,U+nG) gradients, [U+nG,U+2nG) momentum.
+template <int VEC, bool MOMENTUM>
+__device__ __forceinline__ void reduce_apply_record(const HopRecord& r, const HopEntry* __restrict__ ents,
+                                                    const float* __restrict__ stage, int w, int wd, int U, int nG,
+                                                    bool use_g, float lr, float mu, float* __restrict__ X,
+                                                    float* __restrict__ M, int64_t P, int64_t c0, int lane) {
+    const HopEntry* e = ents + r.ent_begin;
+    float* out = X + (int64_t)r.out_row * P + c0;
+    const bool grad = use_g && r.g_stage >= 0;
+    const float* grow = stage + (int64_t)(U + (grad ? r.g_stage : 0)) * w;
+    const float* mrow = stage + (int64_t)(U + nG + (grad ? r.g_stage : 0)) * w;
+    float* mout = MOMENTUM ? (M + (int64_t)r.worker * P + c0) : nullptr;
+    for (int c = lane * VEC; c < wd; c += 32 * VEC) {
+        if constexpr (VEC == 4) {
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int t = 0; t < r.ent_count; ++t) {
+                const HopEntry en = e[t];
+                const float4 v = *reinterpret_cast<const float4*>(stage + (int64_t)en.u * w + c);
+                acc.x = fmaf(en.w, v.x, acc.x); acc.y = fmaf(en.w, v.y, acc.y);
+                acc.z = fmaf(en.w, v.z, acc.z); acc.w = fmaf(en.w, v.w, acc.w);
+            }
+            if (grad) {
+                float4 g = *reinterpret_cast<const float4*>(grow + c);
+                if constexpr (MOMENTUM) {
+                    const float4 m = *reinterpret_cast<const float4*>(mrow + c);
+                    g.x = fmaf(mu, m.x, g.x); g.y = fmaf(mu, m.y, g.y);
+                    g.z = fmaf(mu, m.z, g.z); g.w = fmaf(mu, m.w, g.w);
+                    *reinterpret_cast<float4*>(mout + c) = g;
+                }
+                acc.x = fmaf(-lr, g.x, acc.x); acc.y = fmaf(-lr, g.y, acc.y);
+                acc.z = fmaf(-lr, g.z, acc.z); acc.w = fmaf(-lr, g.w, acc.w);
+            }
+            *reinterpret_cast<float4*>(out + c) = acc;
+        } else {
+            float acc = 0.f;
+            for (int t = 0; t < r.ent_count; ++t) {
+                const HopEntry en = e[t];
+                acc = fmaf(en.w, stage[(int64_t)en.u * w + c], acc);
+            }
+            if (grad) {
+                float g = grow[c];
+                if constexpr (MOMENTUM) {
+                    g = fmaf(mu, mrow[c], g);
+                    mout[c] = g;
+                }
+                acc = fmaf(-lr, g, acc);
+            }
+            out[c] = acc;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// mix_staged: ordinary loads into shared memory, one barrier, compute, one barrier.  Works for any P
+// (VEC = 1 when P is not a multiple of 4).
+template <int VEC, bool MOMENTUM>
+__global__ void __launch_bounds__(kStagedThreads)
+mix_staged_kernel(float* __restrict__ X, float* __restrict__ M, const float* __restrict__ G, int64_t P, int w,
+                  int use_g, float lr, float mu, HopLevelDev lv) {
+    extern __shared__ __align__(16) float smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nG = use_g ? lv.nG : 0;
+    const int64_t tiles = (P + w - 1) / w;
+    for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+        const int64_t c0 = tile * w;
+        const int wd = (int)min((int64_t)w, P - c0);
+        const int per_row = (wd + VEC - 1) / VEC;
+        const int rows = lv.U + nG * (MOMENTUM ? 2 : 1);
+        for (int idx = tid; idx < rows * per_row; idx += kStagedThreads) {
+            const int r = idx / per_row, c = (idx - r * per_row) * VEC;
+            const float* src;
+            if (r < lv.U) src = X + (int64_t)lv.src_row[r] * P;
+            else if (r < lv.U + nG) src = G + (int64_t)lv.grad_workers[r - lv.U] * P;
+            else src = M + (int64_t)lv.grad_workers[r - lv.U - nG] * P;
+            if constexpr (VEC == 4)
+                *reinterpret_cast<float4*>(smem + (int64_t)r * w + c) = *reinterpret_cast<const float4*>(src + c0 + c);
+            else
+                smem[(int64_t)r * w + c] = src[c0 + c];
+        }
+        __syncthreads();
+        for (int a = warp; a < lv.nA; a += kStagedThreads / 32)
+            reduce_apply_record<VEC, MOMENTUM>(lv.recs[a], lv.ents, smem, w, wd, lv.U, nG, use_g != 0, lr, mu, X, M, P, c0, lane);
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// mbarrier / bulk-copy helpers (PTX ISA: mbarrier, cp.async.bulk)
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after kSpinLimit polls so that a lost copy can never hang the GPU.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (it > 64) __nanosleep(64);
+    }
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+// mix_bulk: persistent blocks; warp 0 is the producer (asynchronous bulk copies of every staged row of
+// the next tile, completion counted in bytes on an mbarrier), warps 1..8 consume.  Two stages.
+// Requires P % 4 == 0 and 16-byte aligned base pointers (bulk copies move multiples of 16 bytes).
+template <bool MOMENTUM>
+__global__ void __launch_bounds__(kBulkThreads, 1)
+mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __restrict__ G, int64_t P, int w,
+                int use_g, float lr, float mu, HopLevelDev lv, int32_t* __restrict__ err_word) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw);
+    uint64_t* empty = full + kBulkStages;
+    float* stage0 = reinterpret_cast<float*>(smem_raw + 128);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nG = use_g ? lv.nG : 0;
+    const int rows = lv.U + nG * (MOMENTUM ? 2 : 1);
+    const int64_t stage_floats = (int64_t)rows * w;
+    const int64_t tiles = (P + w - 1) / w;
+    if (tid == 0) {
+        for (int s = 0; s < kBulkStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kConsumerWarps); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 0) {
+        // ---------------- producer
+        int64_t n = 0;
+        bool ok = true;
+        for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++n) {
+            const int s = (int)(n % kBulkStages);
+            const uint32_t ph = (uint32_t)((n / kBulkStages) & 1);
+            if (!mbar_wait(&empty[s], ph ^ 1u)) { ok = false; if (lane == 0) atomicCAS(err_word, 0, ERR_EMPTY_WAIT | (int)(tile & 0xffffff)); break; }
+            const int64_t c0 = tile * w;
+            const int wd = (int)min((int64_t)w, P - c0);
+            const uint32_t bytes = (uint32_t)wd * 4u;
+            if (lane == 0) mbar_expect_tx(&full[s], bytes * (uint32_t)rows);
+            __syncwarp();
+            float* dst = stage0 + s * stage_floats;
+            for (int r = lane; r < rows; r += 32) {
+                const float* src;
+                if (r < lv.U) src = X + (int64_t)lv.src_row[r] * P;
+                else if (r < lv.U + nG) src = G + (int64_t)lv.grad_workers[r - lv.U] * P;
+                else src = M + (int64_t)lv.grad_workers[r - lv.U - nG] * P;
+                bulk_g2s(dst + (int64_t)r * w, src + c0, bytes, &full[s]);
+            }
+        }
+        // drain: do not leave while copies into this block's shared memory are still in flight
+        if (ok) {
+            const int64_t issued = n;
+            for (int64_t m = (issued > kBulkStages ? issued - kBulkStages : 0); m < issued; ++m)
+                mbar_wait(&full[m % kBulkStages], (uint32_t)((m / kBulkStages) & 1));
+        }
+    } else {
+        // ---------------- consumers
+        const int cw = warp - 1;
+        int64_t n = 0;
+        for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++n) {
+            const int s = (int)(n % kBulkStages);
+            const uint32_t ph = (uint32_t)((n / kBulkStages) & 1);
+            if (!mbar_wait(&full[s], ph)) { if (lane == 0) atomicCAS(err_word, 0, ERR_FULL_WAIT | (int)(tile & 0xffffff)); break; }
+            const int64_t c0 = tile * w;
+            const int wd = (int)min((int64_t)w, P - c0);
+            const float* st = stage0 + s * stage_floats;
+            for (int a = cw; a < lv.nA; a += kConsumerWarps)
+                reduce_apply_record<4, MOMENTUM>(lv.recs[a], lv.ents, st, w, wd, lv.U, nG, use_g != 0, lr, mu, X, M, P, c0, lane);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[s]);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11): multipliers and Weyl key increments from the publication.
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1,
+                                              uint32_t (&o)[4]) {
+    constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+        const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+        c0 = hi1 ^ c1 ^ k0; c1 = lo1; c2 = hi0 ^ c3 ^ k1; c3 = lo0;
+        k0 += W0; k1 += W1;
+    }
+    o[0] = c0; o[1] = c1; o[2] = c2; o[3] = c3;
+}
+// Box-Muller on 23-bit uniforms u = (n + 1/2) / 2^23 (exact in float32).
+__device__ __forceinline__ void box_muller(uint32_t ra, uint32_t rb, float& z0, float& z1) {
+    const float u1 = (float)(((ra >> 9) << 1) | 1u) * 5.9604644775390625e-08f;   // (2n+1) * 2^-24
+    const float two_u2 = (float)(((rb >> 9) << 1) | 1u) * 1.1920928955078125e-07f;  // 2 * u2
+    const float rad = sqrtf(-2.0f * logf(u1));
+    float sn, cs;
+    sincospif(two_u2, &sn, &cs);
+    z0 = rad * cs; z1 = rad * sn;
+}
+
+__global__ void __launch_bounds__(256)
+synth_grad_kernel(float* __restrict__ G, int64_t P, HopLevelDev lv, uint32_t k0, uint32_t k1, float sigma, int64_t col_offset) {
+    const int worker = lv.grad_workers[blockIdx.y];
+    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;     // local group of 4 columns
+    const int64_t c = q * 4;
+    if (c >= P) return;
+    uint32_t o[4];
+    const uint64_t gq = (uint64_t)(col_offset / 4 + q);
+    philox4x32_10((uint32_t)gq, (uint32_t)worker, (uint32_t)lv.level, 6u, k0, k1, o);
+    float z[4];
+    box_muller(o[0], o[1], z[0], z[1]);
+    box_muller(o[2], o[3], z[2], z[3]);
+    float* dst = G + (int64_t)worker * P + c;
+    if (c + 4 <= P && (P & 3) == 0) {
+        *reinterpret_cast<float4*>(dst) = make_float4(sigma * z[0], sigma * z[1], sigma * z[2], sigma * z[3]);
+    } else {
+        for (int e = 0; e < 4 && c + e < P; ++e) dst[e] = sigma * z[e];
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Hinge-loss SVM.  One warp per minibatch row: margin = a_r . x_{k,i} accumulated in double (the
+// active-set test y*margin < 1 is then decided as in exact arithmetic up to ~1e-16), reduced with
+// warp shuffles; coef_r = -y_r/B if active else 0.
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__global__ void __launch_bounds__(256)
+svm_margin_csr_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelDev lv, const int64_t* __restrict__ row_ptr,
+                      const int32_t* __restrict__ col, const float* __restrict__ val, const float* __restrict__ y,
+                      int R, int B, float* __restrict__ coef) {
+    const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (gw >= lv.nG * B) return;
+    const int a = gw / B, r = gw - a * B;
+    const int worker = lv.grad_workers[a];
+    const int64_t row = (int64_t)worker * R + (int64_t)(lv.level % (R / B)) * B + r;
+    const float* x = X + ((int64_t)worker * S + lv.level % S) * P;
+    double m = 0.0;
+    for (int64_t t = row_ptr[row] + lane; t < row_ptr[row + 1]; t += 32) m += (double)val[t] * (double)x[col[t]];
+    m = warp_sum(m);
+    if (lane == 0) {
+        const float yy = y[(int64_t)worker * R + (row - (int64_t)worker * R)];
+        coef[(int64_t)worker * B + r] = ((double)yy * m < 1.0) ? -yy / (float)B : 0.f;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+svm_margin_dense_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelDev lv, const float* __restrict__ A,
+                        const float* __restrict__ y, int R, int B, float* __restrict__ coef) {
+    const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (gw >= lv.nG * B) return;
+    const int a = gw / B, r = gw - a * B;
+    const int worker = lv.grad_workers[a];
+    const int64_t row = (int64_t)worker * R + (int64_t)(lv.level % (R / B)) * B + r;
+    const float* x = X + ((int64_t)worker * S + lv.level % S) * P;
+    const float* arow = A + row * P;
+    double m = 0.0;
+    for (int64_t p = lane; p < P; p += 32) m += (double)arow[p] * (double)x[p];
+    m = warp_sum(m);
+    if (lane == 0) {
+        const float yy = y[row];
+        coef[(int64_t)worker * B + r] = ((double)yy * m < 1.0) ? -yy / (float)B : 0.f;
+    }
+}
+
+// g[i][p] = sum_r coef_r * A[r][p]; one thread per column, rows of the minibatch in order.
+__global__ void __launch_bounds__(256)
+svm_dense_grad_kernel(float* __restrict__ G, int64_t P, HopLevelDev lv, const float* __restrict__ A, int R, int B,
+                      const float* __restrict__ coef) {
+    const int worker = lv.grad_workers[blockIdx.y];
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= P) return;
+    const float* a0 = A + ((int64_t)worker * R + (int64_t)(lv.level % (R / B)) * B) * P + p;
+    const float* cf = coef + (int64_t)worker * B;
+    float g = 0.f;
+    for (int r = 0; r < B; ++r) g = fmaf(cf[r], a0[(int64_t)r * P], g);
+    G[(int64_t)worker * P + p] = g;
+}
+
+// Sparse Apply after the dense mix: x_{k+1,i}[col] -= lr * coef_r * val, one warp per row.
+__global__ void __launch_bounds__(256)
+svm_csr_apply_kernel(float* __restrict__ X, int64_t P, int S, float lr, HopLevelDev lv, const int64_t* __restrict__ row_ptr,
+                     const int32_t* __restrict__ col, const float* __restrict__ val, int R, int B,
+                     const float* __restrict__ coef) {
+    const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (gw >= lv.nG * B) return;
+    const int a = gw / B, r = gw - a * B;
+    const int worker = lv.grad_workers[a];
+    const float cf = coef[(int64_t)worker * B + r];
+    if (cf == 0.f) return;
+    const int64_t row = (int64_t)worker * R + (int64_t)(lv.level % (R / B)) * B + r;
+    float* x = X + ((int64_t)worker * S + (lv.level + 1) % S) * P;
+    const float scale = -lr * cf;
+    for (int64_t t = row_ptr[row] + lane; t < row_ptr[row + 1]; t += 32) atomicAdd(x + col[t], scale * val[t]);
+}
+
+size_t staged_smem(const HopLaunchCfg& c, const HopLevelDev& lv) {
+    const int nG = c.use_g ? lv.nG : 0;
+    const int rows = lv.U + nG * (c.mu != 0.f ? 2 : 1);
+    return (size_t)rows * c.tile_w * sizeof(float);
+}
+
+}  // namespace
+
+int hop_mix_smem_budget(int kernel) { return kernel == HOP_MIX_BULK ? (227 * 1024 - 128) : 100 * 1024; }
+int hop_mix_stages(int kernel) { return kernel == HOP_MIX_BULK ? kBulkStages : 1; }
+
+int hop_launch_mix_staged(const HopLaunchCfg& c, const HopLevelDev& lv) {
+    if (lv.nA == 0) return 0;
+    const size_t smem = staged_smem(c, lv);
+    const int64_t tiles = (c.P + c.tile_w - 1) / c.tile_w;
+    const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(8, (200 * 1024) / std::max<size_t>(smem, 1)));
+    const int grid = (int)std::min<int64_t>(tiles, (int64_t)c.sm_count * per_sm);
+    const bool vec = (c.P % 4 == 0) && (c.tile_w % 4 == 0);
+    const bool mom = c.mu != 0.f;
+    cudaStream_t st = (cudaStream_t)c.stream;
+    cudaError_t e = cudaSuccess;
+#define HOP_LAUNCH_STAGED(V, MO)                                                                              \
+    do {                                                                                                      \
+        e = cudaFuncSetAttribute(mix_staged_kernel<V, MO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        if (e == cudaSuccess)                                                                                 \
+            mix_staged_kernel<V, MO><<<grid, kStagedThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, lv); \
+    } while (0)
+    if (vec && mom) HOP_LAUNCH_STAGED(4, true);
+    else if (vec) HOP_LAUNCH_STAGED(4, false);
+    else if (mom) HOP_LAUNCH_STAGED(1, true);
+    else HOP_LAUNCH_STAGED(1, false);
+#undef HOP_LAUNCH_STAGED
+    if (e != cudaSuccess) return (int)e;
+    return (int)cudaGetLastError();
+}
+
+int hop_launch_mix_bulk(const HopLaunchCfg& c, const HopLevelDev& lv) {
+    if (lv.nA == 0) return 0;
+    const int nG = c.use_g ? lv.nG : 0;
+    const int rows = lv.U + nG * (c.mu != 0.f ? 2 : 1);
+    const size_t smem = 128 + (size_t)kBulkStages * rows * c.tile_w * sizeof(float);
+    const int64_t tiles = (c.P + c.tile_w - 1) / c.tile_w;
+    const int grid = (int)std::min<int64_t>(tiles, (int64_t)c.sm_count);
+    cudaStream_t st = (cudaStream_t)c.stream;
+    cudaError_t e;
+    if (c.mu != 0.f) {
+        e = cudaFuncSetAttribute(mix_bulk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+        mix_bulk_kernel<true><<<grid, kBulkThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, lv, c.err_word);
+    } else {
+        e = cudaFuncSetAttribute(mix_bulk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+        mix_bulk_kernel<false><<<grid, kBulkThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, lv, c.err_word);
+    }
+    return (int)cudaGetLastError();
+}
+
+int hop_launch_synth_grad(const HopLaunchCfg& c, const HopLevelDev& lv, uint64_t seed, float sigma, int64_t col_offset) {
+    if (lv.nG == 0) return 0;
+    const int64_t groups = (c.P + 3) / 4;
+    dim3 grid((unsigned)((groups + 255) / 256), (unsigned)lv.nG);
+    synth_grad_kernel<<<grid, 256, 0, (cudaStream_t)c.stream>>>(c.G, c.P, lv, (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), sigma, col_offset);
+    return (int)cudaGetLastError();
+}
+
+int hop_launch_svm_dense(const HopLaunchCfg& c, const HopLevelDev& lv, const float* A, const float* y,
+                         int32_t R, int32_t B, float* coef) {
+    if (lv.nG == 0) return 0;
+    const int warps = lv.nG * B;
+    svm_margin_dense_kernel<<<(warps * 32 + 255) / 256, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.P, c.s + 1, lv, A, y, R, B, coef);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return (int)e;
+    dim3 grid((unsigned)((c.P + 255) / 256), (unsigned)lv.nG);
+    svm_dense_grad_kernel<<<grid, 256, 0, (cudaStream_t)c.stream>>>(c.G, c.P, lv, A, R, B, coef);
+    return (int)cudaGetLastError();
+}
+
+int hop_launch_svm_csr_coef(const HopLaunchCfg& c, const HopLevelDev& lv, const int64_t* row_ptr, const int32_t* col,
+                            const float* val, const float* y, int32_t R, int32_t B, float* coef) {
+    if (lv.nG == 0) return 0;
+    const int warps = lv.nG * B;
+    svm_margin_csr_kernel<<<(warps * 32 + 255) / 256, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.P, c.s + 1, lv, row_ptr, col, val, y, R, B, coef);
+    return (int)cudaGetLastError();
+}
+
+int hop_launch_svm_csr_apply(const HopLaunchCfg& c, const HopLevelDev& lv, const int64_t* row_ptr, const int32_t* col,
+                             const float* val, int32_t R, int32_t B, const float* coef) {
+    if (lv.nG == 0) return 0;
+    const int warps = lv.nG * B;
+    svm_csr_apply_kernel<<<(warps * 32 + 255) / 256, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.P, c.s + 1, c.lr, lv, row_ptr, col, val, R, B, coef);
+    return (int)cudaGetLastError();
+}

@@ -61,14 +61,20 @@ def csr_to_lists(in_ptr, in_idx) -> list[list[int]]:
 
 
 # ---------------------------------------------------------------- graph constructors
+# Every constructor returns in-neighbour lists (self included) in ascending id order: that is the
+# order in which trace records list the consumed neighbours.
+def _canon(n_in):
+    return [sorted(set(nb)) for nb in n_in]
+
+
 def ring(n: int) -> list[list[int]]:
     """Bidirectional ring: N_in(i) = {i, i-1, i+1}."""
-    return [[i, (i - 1) % n, (i + 1) % n] for i in range(n)]
+    return _canon([[i, (i - 1) % n, (i + 1) % n] for i in range(n)])
 
 
 def ring_chords(n: int, chord: int) -> list[list[int]]:
     """Ring plus +-chord links: N_in(i) = {i, i+-1, i+-chord}."""
-    return [[i, (i - 1) % n, (i + 1) % n, (i - chord) % n, (i + chord) % n] for i in range(n)]
+    return _canon([[i, (i - 1) % n, (i + 1) % n, (i - chord) % n, (i + chord) % n] for i in range(n)])
 
 
 def torus(nx: int, ny: int) -> list[list[int]]:
@@ -79,7 +85,7 @@ def torus(nx: int, ny: int) -> list[list[int]]:
             out.append([y * nx + x,
                         y * nx + (x - 1) % nx, y * nx + (x + 1) % nx,
                         ((y - 1) % ny) * nx + x, ((y + 1) % ny) * nx + x])
-    return out
+    return _canon(out)
 
 
 def complete(n: int) -> list[list[int]]:
@@ -88,12 +94,12 @@ def complete(n: int) -> list[list[int]]:
 
 def directed_cycle(n: int) -> list[list[int]]:
     """i receives from i-1 only (plus itself)."""
-    return [[i, (i - 1) % n] for i in range(n)]
+    return _canon([[i, (i - 1) % n] for i in range(n)])
 
 
 def ring_based(n: int) -> list[list[int]]:
     """Ring where every node is also linked to the most distant node (paper Fig. 'Graphs used in experiments' (2))."""
-    return [[i, (i - 1) % n, (i + 1) % n, (i + n // 2) % n] for i in range(n)]
+    return _canon([[i, (i - 1) % n, (i + 1) % n, (i + n // 2) % n] for i in range(n)])
 
 
 def double_ring(n: int) -> list[list[int]]:
@@ -104,7 +110,7 @@ def double_ring(n: int) -> list[list[int]]:
     for g in range(2):
         for i in range(h):
             out.append([g * h + j for j in base[i]] + [(1 - g) * h + i])
-    return out
+    return _canon(out)
 
 
 def _strongly_connected(n_in: list[list[int]]) -> bool:
@@ -141,7 +147,7 @@ def random_regular_digraph(n: int, deg: int, rng: np.random.Generator) -> list[l
             perms.append(p)
         n_in = [[i] + [int(p[i]) for p in perms] for i in range(n)]
         if _strongly_connected(n_in):
-            return n_in
+            return _canon(n_in)
 
 
 # ---------------------------------------------------------------- workload container

@@ -1,0 +1,114 @@
+"""Production protocol simulator (C++, queue-free formulation) against the oracle (Python, literal
+queues): traces must be bit-identical.  CPU only: hop_sim_run touches no GPU."""
+import itertools
+
+import numpy as np
+import pytest
+
+from oracle import protocol as op
+from paper_1902_01064_b200 import hop, inputs
+
+KEYS = ("op", "ptr", "nbr", "ver", "num", "den")
+
+
+def both(n_in, ticks, iters, s, b, max_ig, max_skip, mode):
+    ptr, idx = inputs.graph_to_csr(n_in)
+    n_in = inputs.csr_to_lists(ptr, idx)                 # records list neighbours in ascending id order
+    h = hop.Hop(ptr, idx, len(n_in), 8, s, b, max_skip)
+    h.set_option(hop.OPT_MAX_IG, 0 if max_ig is None else max_ig)
+    h.set_option(hop.OPT_WEIGHT_MODE, mode)
+    got = h.sim_run(ticks, iters).to_arrays()
+    want_tr = op.simulate(n_in, ticks, iters, s, b, max_ig, max_skip, mode)
+    want = want_tr.to_arrays()
+    h.close()
+    return got, want, want_tr.makespan
+
+
+def assert_same(got, want, makespan, ctx=""):
+    for k in KEYS:
+        assert np.array_equal(got[k], want[k]), (k, ctx)
+    assert got["makespan"] == makespan, ctx
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_configs_bit_exact(cfg):
+    w = inputs.make_workload(cfg, P=64 if cfg == 1 else 256)
+    got, want, mk = both(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode)
+    assert_same(got, want, mk, cfg)
+    assert (got["op"] != op.IDLE).sum() > 0
+
+
+def _enumerate(name, n_in, iters, values, combos):
+    N = len(n_in)
+    count = 0
+    for flat in itertools.product(values, repeat=N * iters):
+        ticks = np.asarray(flat, np.uint64).reshape(N, iters)
+        for (s, b, max_skip) in combos:
+            if any(b >= len(nb) for nb in n_in) or max_skip > s + 1:
+                continue
+            max_ig = max(1, s)
+            got, want, mk = both(n_in, ticks, iters, s, b, max_ig, max_skip, op.STALE_LINEAR)
+            assert_same(got, want, mk, (name, flat, s, b, max_skip))
+            count += 1
+    return count
+
+
+ALL_COMBOS = [(s, b, k) for s in (0, 1, 2) for b in (0, 1) for k in (0, 1, 2)]
+
+
+def test_exhaustive_three_workers_two_iterations():
+    for name, n_in in inputs.small_cases()[:2]:
+        assert _enumerate(name, n_in, 2, (1, 2, 3), ALL_COMBOS) > 5000
+
+
+def test_exhaustive_three_workers_three_iterations():
+    # 2^9 tick tables x all protocol settings, two tick alphabets
+    for name, n_in in inputs.small_cases()[:2]:
+        _enumerate(name, n_in, 3, (1, 2), ALL_COMBOS)
+        _enumerate(name, n_in, 3, (1, 3), [(1, 1, 2), (2, 0, 2), (0, 1, 1)])
+
+
+def test_exhaustive_four_workers():
+    for name, n_in in inputs.small_cases()[2:]:
+        _enumerate(name, n_in, 2, (1, 2), ALL_COMBOS)
+        _enumerate(name, n_in, 3, (1, 2), [(1, 1, 2), (2, 0, 1)])
+
+
+def test_random_graphs_long_runs_with_ties_and_skips():
+    rng = np.random.default_rng(42)
+    for trial in range(60):
+        N = int(rng.integers(3, 12))
+        n_in = [{i, (i - 1) % N} for i in range(N)]
+        for _ in range(int(rng.integers(0, 3 * N))):
+            a, c = rng.integers(0, N, 2)
+            n_in[int(a)].add(int(c))
+        n_in = [sorted(x) for x in n_in]
+        s = int(rng.integers(0, 4))
+        b = int(rng.integers(0, min(len(x) for x in n_in)))
+        max_skip = int(rng.integers(0, s + 2))
+        max_ig = int(rng.integers(1, 5))
+        iters = 25
+        ticks = rng.choice([1, 1, 1, 2, 5], size=(N, iters)).astype(np.uint64)
+        if trial % 3 == 0:
+            ticks[int(rng.integers(0, N)), :] *= 4          # deterministic straggler
+        mode = int(rng.integers(0, 2))
+        try:
+            want_tr = op.simulate(n_in, ticks, iters, s, b, max_ig, max_skip, mode)
+        except op.Deadlock:
+            ptr, idx = inputs.graph_to_csr(n_in)
+            h = hop.Hop(ptr, idx, N, 8, s, b, max_skip)
+            h.set_option(hop.OPT_MAX_IG, max_ig)
+            with pytest.raises(hop.HopError) as e:
+                h.sim_run(ticks, iters)
+            assert e.value.code == hop.E_DEADLOCK
+            continue
+        got, want, mk = both(n_in, ticks, iters, s, b, max_ig, max_skip, mode)
+        assert_same(got, want, mk, trial)
+
+
+def test_unbounded_gap_without_tokens():
+    n_in = inputs.complete(3)
+    ticks = np.ones((3, 12), np.uint64)
+    ticks[0, 0] = 10 ** 12
+    got, want, mk = both(n_in, ticks, 12, 0, 1, None, 0, op.UNIFORM)
+    assert_same(got, want, mk)
