@@ -1,0 +1,280 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element.
+
+Tolerances (float32 path against a float64 oracle): max|delta| <= 1e-6 * max|x| after one level,
+<= 1e-4 * max|x| after a full run; traces are compared bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import philox, protocol as op, update as up
+from paper_1902_01064_b200 import hop, inputs
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+TOL_STEP, TOL_RUN = 1e-6, 1e-4
+KEYS = ("op", "ptr", "nbr", "ver", "num", "den")
+
+
+class GpuRun:
+    """Device buffers (torch, plumbing only) + a configured context for a workload."""
+
+    def __init__(self, w, mix_kernel=hop.MIX_AUTO, x0=None, external_G=None):
+        self.w = w
+        S = w.s + 1
+        self.X = torch.zeros((w.N, S, w.P), dtype=torch.float32, device=DEV)
+        self.M = torch.zeros((w.N, w.P), dtype=torch.float32, device=DEV) if w.momentum else None
+        self.G = None if w.grad_mode == inputs.GRAD_SVM_CSR else torch.zeros((w.N, w.P), dtype=torch.float32, device=DEV)
+        self.h = hop.from_workload(w, mix_kernel)
+        if external_G is not None:
+            self.h.set_option(hop.OPT_GRAD_MODE, hop.GRAD_EXTERNAL)
+        self.external_G = external_G
+        self.h.bind_buffers(self.X, self.M, self.G, torch.cuda.current_stream().cuda_stream)
+        if w.grad_mode == inputs.GRAD_SVM_DENSE:
+            self.A = torch.from_numpy(w.svm.dense).to(DEV)
+            self.y = torch.from_numpy(w.svm.y).to(DEV)
+            self.h.bind_svm_dense(self.A, self.y, w.svm.rows_per_worker, w.svm.batch)
+        elif w.grad_mode == inputs.GRAD_SVM_CSR:
+            self.rp = torch.from_numpy(w.svm.row_ptr).to(DEV)
+            self.col = torch.from_numpy(w.svm.col).to(DEV)
+            self.val = torch.from_numpy(w.svm.val).to(DEV)
+            self.y = torch.from_numpy(w.svm.y).to(DEV)
+            self.h.bind_svm_csr(self.rp, self.col, self.val, self.y, w.svm.rows_per_worker, w.svm.batch)
+        self.trace = self.h.sim_run(w.ticks, w.iters)
+        self.h.load_trace(self.trace)
+        self.x0 = np.tile(w.p0(), (w.N, 1)) if x0 is None else x0
+        for i in range(w.N):
+            self.h.write_params(i, 0, self.x0[i])
+
+    def run(self, levels):
+        for k in range(levels):
+            if self.external_G is not None:
+                self.G.copy_(torch.from_numpy(self.external_G[k]))
+            self.h.step()
+        assert self.h.read_status() == 0
+        return [self.h.read_params(i) for i in range(self.w.N)]
+
+
+def oracle_grad_fn(w, cols=None, external_G=None):
+    if external_G is not None:
+        return up.GradExternal(external_G if cols is None else external_G[:, :, cols])
+    if w.grad_mode == inputs.GRAD_SYNTHETIC:
+        return up.GradSynthetic(w.grad_seed, w.sigma, np.arange(w.P) if cols is None else cols)
+    if w.grad_mode == inputs.GRAD_SVM_DENSE:
+        return up.GradSvmDense(w.svm.dense, w.svm.y, w.svm.batch)
+    return up.GradSvmCsr(w.svm.row_ptr, w.svm.col, w.svm.val, w.svm.y, w.svm.rows_per_worker, w.svm.batch)
+
+
+def oracle_run(w, x0, levels, cols=None, external_G=None):
+    tr = op.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode).to_arrays()
+    xs = x0.astype(np.float64) if cols is None else x0[:, cols].astype(np.float64)
+    X, newest = up.run_updates(tr, w.N, w.lr, w.momentum, xs, oracle_grad_fn(w, cols, external_G), levels=levels, s=w.s)
+    return tr, [X[(i, newest[i])] for i in range(w.N)], newest
+
+
+def check(w, levels, tol, mix_kernel=hop.MIX_AUTO, perturb=False, cols=None, external_G=None):
+    x0 = np.tile(w.p0(), (w.N, 1))
+    if perturb:
+        x0 = np.stack([w.p0() + w.perturbation(i) for i in range(w.N)])
+    g = GpuRun(w, mix_kernel, x0, external_G)
+    got = g.run(levels)
+    tr, want, newest = oracle_run(w, x0, levels, cols, external_G)
+    gt = g.trace.to_arrays()
+    for k in KEYS:
+        assert np.array_equal(gt[k], tr[k]), k                                  # traces bit-exact
+    scale = max(1e-30, max(np.abs(x).max() for x in want))
+    worst = 0.0
+    for i in range(w.N):
+        assert g.h.newest_version(i) == newest[i]
+        a = got[i].astype(np.float64) if cols is None else got[i][cols].astype(np.float64)
+        worst = max(worst, np.abs(a - want[i]).max())
+    assert worst <= tol * scale, (worst, scale)
+    g.h.close()
+    return worst / scale
+
+
+KERNELS = [hop.MIX_STAGED, hop.MIX_BULK]
+
+
+# ------------------------------------------------------------------ configuration 1: dense SVM, 4 workers
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_cfg1_full_run_and_one_step(kernel):
+    w = inputs.make_workload(1)
+    check(w, w.iters, TOL_RUN, kernel)
+    check(w, 1, TOL_STEP, kernel, perturb=True)
+    check(w, 5, TOL_RUN, kernel, perturb=True)
+
+
+# ------------------------------------------------------------------ configuration 2: CSR SVM, 16 workers
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_cfg2_reduced_full_run(kernel):
+    w = inputs.make_workload(2, P=8192)
+    check(w, w.iters, TOL_RUN, kernel)
+    check(w, 1, TOL_STEP, kernel, perturb=True)
+
+
+def test_cfg2_full_size_first_levels():
+    w = inputs.make_workload(2)
+    check(w, 1, TOL_STEP, perturb=True)
+    check(w, 6, TOL_RUN)
+
+
+# ------------------------------------------------------------------ configuration 3: momentum + skipping
+@pytest.mark.parametrize("kernel,P", [(hop.MIX_STAGED, 5000), (hop.MIX_BULK, 5000), (hop.MIX_STAGED, 4999),
+                                      (hop.MIX_BULK, 132), (hop.MIX_STAGED, 3)])
+def test_cfg3_reduced_full_run(kernel, P):
+    w = inputs.make_workload(3, P=P)
+    check(w, w.iters, TOL_RUN, kernel)
+    check(w, 1, TOL_STEP, kernel, perturb=True)
+
+
+def test_cfg3_full_size_sampled_columns():
+    w = inputs.make_workload(3)
+    g = GpuRun(w)
+    tile = g.h.level_stats(0)["tile_w"]
+    cols = np.unique(np.concatenate([np.arange(0, w.P, 997), np.arange(tile - 2, w.P, 50 * tile),
+                                     np.arange(tile, w.P, 50 * tile), [w.P - 1, w.P - 2, w.P - 5]]))
+    g.h.close()
+    check(w, w.iters, TOL_RUN, cols=cols)
+
+
+# ------------------------------------------------------------------ configuration 4: 64 workers, s=4, b=2
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_cfg4_reduced_full_run(kernel):
+    w = inputs.make_workload(4, P=3000)
+    check(w, w.iters, TOL_RUN, kernel)
+    check(w, 1, TOL_STEP, kernel, perturb=True)
+
+
+def test_cfg4_full_size_sampled_columns():
+    w = inputs.make_workload(4)
+    free, _ = torch.cuda.mem_get_info()
+    if free < 50 * 2 ** 30:
+        pytest.skip("needs ~42 GB of device memory")
+    cols = np.unique(np.concatenate([np.arange(0, w.P, 25013), np.arange(127, w.P, 128 * 4001),
+                                     np.arange(128, w.P, 128 * 4001), [w.P - 1, w.P - 4]]))
+    check(w, w.iters, TOL_RUN, cols=cols)
+
+
+# ------------------------------------------------------------------ configuration 5: complete graph, 128 workers
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_cfg5_reduced_full_run(kernel):
+    w = inputs.make_workload(5, P=1536)
+    check(w, w.iters, TOL_RUN, kernel)
+    check(w, 1, TOL_STEP, kernel, perturb=True)
+
+
+def test_cfg5_full_size_sampled_columns_first_levels():
+    w = inputs.make_workload(5)
+    cols = np.unique(np.concatenate([np.arange(0, w.P, 40009), [w.P - 1, w.P - 3, 127, 128, 255, 256]]))
+    check(w, 4, TOL_RUN, cols=cols)
+
+
+# ------------------------------------------------------------------ kernels in isolation / edge cases
+def test_synthetic_gradient_kernel_matches_philox_box_muller():
+    w = inputs.make_workload(3, P=10007)
+    g = GpuRun(w, hop.MIX_STAGED)
+    g.h.step()
+    torch.cuda.synchronize()
+    G = g.G.cpu().numpy()
+    tr = g.trace.to_arrays()
+    for i in range(w.N):
+        if tr["op"][0, i] == op.NORMAL:
+            want = philox.synthetic_gradient(w.grad_seed, i, 0, np.arange(w.P), w.sigma)
+            assert np.abs(G[i] - want).max() <= 2e-6 * w.sigma * 6
+    g.h.close()
+
+
+def test_external_gradients_and_tiny_shapes():
+    rng = np.random.default_rng(0)
+    for (N, P, s) in [(1, 1, 0), (2, 4, 0), (3, 7, 1), (5, 33, 2), (6, 260, 0)]:
+        n_in = inputs.complete(N) if N < 4 else inputs.ring(N)
+        ptr, idx = inputs.graph_to_csr(n_in)
+        iters = 6
+        w = inputs.Workload(0, "tiny", N, P, iters, s=s, b=0, max_skip=0, max_ig=max(1, s), lr=0.25, momentum=0.5,
+                            weight_mode=inputs.STALE_LINEAR, grad_mode=inputs.GRAD_EXTERNAL, in_ptr=ptr, in_idx=idx,
+                            ticks=rng.integers(1, 9, size=(N, iters)).astype(np.uint64))
+        w._p0 = rng.standard_normal(P).astype(np.float32)
+        G = rng.standard_normal((iters, N, P)).astype(np.float32)
+        for kernel in ([hop.MIX_STAGED, hop.MIX_BULK] if P % 4 == 0 else [hop.MIX_STAGED]):
+            check(w, iters, TOL_RUN, kernel, perturb=True, external_G=G)
+
+
+def test_in_place_ring_hazard_single_slot_and_stale_reads():
+    # s = 0: one slot per worker, every level overwrites what the neighbours read in that level.
+    rng = np.random.default_rng(1)
+    for s, P in [(0, 1000), (1, 1000), (3, 1000), (0, 20000)]:
+        n_in = inputs.ring_chords(12, 5)
+        ptr, idx = inputs.graph_to_csr(n_in)
+        iters = 12
+        ticks = rng.choice([1, 1, 7], size=(12, iters)).astype(np.uint64)     # stragglers -> oldest versions consumed
+        w = inputs.Workload(0, "hazard", 12, P, iters, s=s, b=0, max_skip=0, max_ig=max(1, s), lr=0.1, momentum=0.0,
+                            weight_mode=inputs.STALE_LINEAR, grad_mode=inputs.GRAD_SYNTHETIC, in_ptr=ptr, in_idx=idx,
+                            ticks=ticks, grad_seed=77)
+        w._p0 = rng.standard_normal(P).astype(np.float32)
+        tr = op.simulate(w.n_in, ticks, iters, s, 0, w.max_ig, 0, w.weight_mode)
+        if s > 0:
+            oldest = sum(1 for (k, i), rec in tr.rec.items() for (j, v, _) in rec if j != i and v == k - s)
+            assert oldest > 0, "no slot is read in the level that overwrites it: test is vacuous"
+        for kernel in KERNELS:
+            check(w, iters, TOL_RUN, kernel, perturb=True)
+
+
+def test_streaming_levels_equal_preloaded_trace_bitwise():
+    w = inputs.make_workload(3, P=2048, iters=40)
+    a = GpuRun(w)
+    ref = a.run(w.iters)
+    b = GpuRun(w)
+    tr = b.trace.to_arrays()
+    b.h.set_level(0)
+    probe = np.zeros(16, np.float32)
+    N = w.N
+    for k in range(w.iters):
+        lo, hi = tr["ptr"][k * N], tr["ptr"][(k + 1) * N]
+        ptr = (tr["ptr"][k * N:(k + 1) * N + 1] - lo).astype(np.int64)
+        b.h.step_host(np.ascontiguousarray(tr["op"][k]), ptr, np.ascontiguousarray(tr["nbr"][lo:hi]),
+                      np.ascontiguousarray(tr["ver"][lo:hi]), np.ascontiguousarray(tr["num"][lo:hi]),
+                      np.ascontiguousarray(tr["den"][k]), probe)
+    for i in range(N):
+        assert np.array_equal(ref[i], b.h.read_params(i))
+    assert np.array_equal(probe, ref[0][:16])
+    a.h.close()
+    b.h.close()
+
+
+def test_checkpoint_resume_is_bitwise():
+    w = inputs.make_workload(3, P=1024, iters=30)
+    a = GpuRun(w)
+    ref = a.run(w.iters)
+    b = GpuRun(w)
+    b.run(17)
+    torch.cuda.synchronize()
+    ringX, ringM = b.X.clone(), b.M.clone()
+    c = GpuRun(w)
+    c.X.copy_(ringX)
+    c.M.copy_(ringM)
+    c.h.set_level(17)
+    for k in range(17, w.iters):
+        c.h.step()
+    for i in range(w.N):
+        assert np.array_equal(ref[i], c.h.read_params(i))
+    for x in (a, b, c):
+        x.h.close()
+
+
+def test_malformed_traces_are_rejected_on_the_host():
+    w = inputs.make_workload(4, P=64, iters=8)
+    g = GpuRun(w)
+    good = g.trace.to_arrays()
+
+    def load(mut):
+        t = {k: good[k].copy() for k in KEYS}
+        mut(t)
+        with pytest.raises(hop.HopError) as e:
+            g.h.load_trace(hop.Trace.from_arrays(*[t[k] for k in KEYS]))
+        assert e.value.code == hop.E_TRACE
+    load(lambda t: t["ver"].__setitem__(5, t["ver"][5] - 9))                  # older than the staleness window
+    load(lambda t: t["nbr"].__setitem__(1, (t["nbr"][1] + 1) % 64))           # likely not an in-neighbour / duplicate
+    load(lambda t: t["den"].__setitem__((3, 3), t["den"][3, 3] + 1))          # weights do not sum up
+    load(lambda t: t["op"].__setitem__((2, 0), 7))                            # unknown op
+    g.h.load_trace(g.trace)
+    g.h.close()
