@@ -1,0 +1,338 @@
+#!/usr/bin/env python
+"""Benchmark of the Hop hot path: worker-iterations/s on B200 and the mix-update kernel's HBM roofline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
+
+A step is one logical iteration (level) of the whole hot path for all workers: gradient kernel(s) on
+x_k, fused gather-mix-update into x_{k+1}, sparse apply (CSR SVM).  The default workload is
+configuration 4: 64 workers on a seeded random 6-regular digraph, P = 25.6M float32 parameters, s = 4
+(32.8 GB of replicas), b = 2, synthetic gradients, 50 levels; with K > 50 the trace is replayed.
+With N > 1 (one process per GPU under torch.distributed.run) the parameter index is sharded across the
+ranks (strong scaling): mixing is separable by column, so there is no data-path collective.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "worker_iterations_per_s"
+UNIT = "worker-iterations/s"
+PROBE = 1024
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the mix-update kernel from the ncu capture
+# summarised under profiles/ (a smaller P scaled by columns), or None when the kernel changed since.
+NCU_TRAFFIC = {}
+
+
+def shard_columns(P: int, n: int, r: int, unit: int = 128):
+    """Contiguous column range of rank r out of n, boundaries on multiples of `unit`."""
+    blocks = (P + unit - 1) // unit
+    lo = (blocks * r // n) * unit
+    hi = min(P, (blocks * (r + 1) // n) * unit)
+    return lo, hi
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.stop_flag, self.samples, self.reasons = index, False, [], set()
+        self.max_mhz = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {nv.nvmlClocksEventReasonHwSlowdown: "hw_slowdown", nv.nvmlClocksEventReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                 nv.nvmlClocksEventReasonSwThermalSlowdown: "sw_thermal_slowdown", nv.nvmlClocksEventReasonSwPowerCap: "sw_power_cap"}
+        while not self.stop_flag:
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.dev, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.dev)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def result(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def oracle_sample(w, budget_cols=131072, levels=6):
+    """The CPU oracle, as it stands, on a bounded sample of the workload: the full protocol simulation
+    plus `levels` levels of the fp64 update rules on `budget_cols` columns (the synthetic-gradient path
+    is separable by column, so work scales linearly in columns).  Returns (worker-iterations/s scaled
+    to the full parameter count, description)."""
+    from oracle import protocol, update
+    t0 = time.perf_counter()
+    tr = protocol.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode).to_arrays()
+    t_sim = time.perf_counter() - t0
+    levels = min(levels, w.iters)
+    if w.grad_mode == 1:
+        C = min(w.P, budget_cols)
+        cols = np.arange(C, dtype=np.int64) * (w.P // C)
+        x0 = np.tile(w.p0()[cols].astype(np.float64), (w.N, 1))
+        grad = update.GradSynthetic(w.grad_seed, w.sigma, cols)
+    else:
+        C = w.P
+        x0 = np.tile(w.p0().astype(np.float64), (w.N, 1))
+        grad = (update.GradSvmDense(w.svm.dense, w.svm.y, w.svm.batch) if w.grad_mode == 2 else
+                update.GradSvmCsr(w.svm.row_ptr, w.svm.col, w.svm.val, w.svm.y, w.svm.rows_per_worker, w.svm.batch))
+    t0 = time.perf_counter()
+    update.run_updates(tr, w.N, w.lr, w.momentum, x0, grad, levels=levels, s=w.s)
+    t_upd = time.perf_counter() - t0
+    n_wi = int((tr["op"][:levels] == 1).sum())
+    total_wi = int((tr["op"] == 1).sum())
+    # time for the whole job at full P: protocol once + update rules scaled by columns and levels
+    per_wi = t_upd / n_wi * (w.P / C)
+    value = total_wi / (t_sim + per_wi * total_wi)
+    desc = (f"protocol simulation of all {w.iters} levels ({t_sim:.2f} s) + fp64 update rules for the first {levels} levels on "
+            f"{C} of {w.P} columns ({t_upd:.2f} s), scaled linearly in columns and levels")
+    return value, desc
+
+
+def run_reference(args):
+    """CPU oracle arm: same config, metric and unit; each step is a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_1902_01064_b200 import inputs
+    w = inputs.make_workload(args.config)
+    vals = []
+    steps, warm = max(1, min(args.steps, 3)), min(args.warmup, 1)
+    for it in range(warm + steps):
+        v, desc = oracle_sample(w, budget_cols=32768, levels=2)
+        if it >= warm:
+            vals.append(v)
+    value = float(np.mean(vals))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * (w.N / value), "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"config {args.config}: {w.name}", "N": w.N, "P": w.P, "s": w.s, "b": w.b, "levels": w.iters},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=4)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--P", type=int, default=None, help="override the parameter count (profiling on a small case)")
+    ap.add_argument("--mix-kernel", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_1902_01064_b200 import build as _b
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if rank == 0:
+        _b.build()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the Hop hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    from paper_1902_01064_b200 import hop, inputs
+
+    w = inputs.make_workload(args.config, P=args.P)
+    P_global = w.P
+    lo, hi = shard_columns(P_global, world, rank)
+    p0 = w.p0()[lo:hi].copy()
+    w.P = hi - lo
+    dev = torch.device("cuda", local)
+    S = w.s + 1
+    X = torch.zeros((w.N, S, w.P), dtype=torch.float32, device=dev)
+    M = torch.zeros((w.N, w.P), dtype=torch.float32, device=dev) if w.momentum else None
+    G = None if w.grad_mode == inputs.GRAD_SVM_CSR else torch.zeros((w.N, w.P), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    h = hop.from_workload(w, args.mix_kernel)
+    h.set_option(hop.OPT_COL_OFFSET, lo)
+    h.bind_buffers(X, M, G, stream.cuda_stream)
+    keep = []
+    if w.grad_mode == inputs.GRAD_SVM_DENSE:
+        keep = [torch.from_numpy(w.svm.dense).to(dev), torch.from_numpy(w.svm.y).to(dev)]
+        h.bind_svm_dense(keep[0], keep[1], w.svm.rows_per_worker, w.svm.batch)
+    elif w.grad_mode == inputs.GRAD_SVM_CSR:
+        keep = [torch.from_numpy(a).to(dev) for a in (w.svm.row_ptr, w.svm.col, w.svm.val, w.svm.y)]
+        h.bind_svm_csr(*keep, w.svm.rows_per_worker, w.svm.batch)
+    t0 = time.perf_counter()
+    trace = h.sim_run(w.ticks, w.iters)
+    sim_ms = 1e3 * (time.perf_counter() - t0)
+    h.load_trace(trace)
+    tr = trace.to_arrays()
+    wi_per_level = (tr["op"] == 1).sum(axis=1)
+    p0_dev = torch.from_numpy(p0).to(dev)
+
+    def reset():
+        X.zero_()
+        X[:, 0, :] = p0_dev
+        if M is not None:
+            M.zero_()
+        h.set_level(0)
+        torch.cuda.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def run_levels(n, first=0):
+        """n consecutive levels starting at trace level `first` (mod the trace length)."""
+        done = 0
+        k = first % w.iters
+        h.set_level(k)
+        wi = 0
+        while done < n:
+            if k == w.iters:
+                k = 0
+                h.set_level(0)
+            h.step()
+            wi += int(wi_per_level[k])
+            k += 1
+            done += 1
+        return wi
+
+    # ---- warm-up, then the timed region: exactly K steps between two events on the launching stream
+    reset()
+    run_levels(max(3, args.warmup))
+    reset()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = h.launch_count()
+    h.timing_enable(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    wi = run_levels(args.steps)
+    e1.record(stream)
+    barrier()
+    sampler.stop_flag = True
+    ms = e0.elapsed_time(e1)
+    tim = h.timing_read()
+    h.timing_enable(False)
+    launches = h.launch_count() - launches0
+    assert h.read_status() == 0
+    sampler.join(timeout=1.0)
+    if dist is not None:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = wi / (ms * 1e-3)
+
+    # ---- end to end: each level's records handed over from host memory, probe read back
+    e2e = None
+    if not args.no_e2e:
+        reset()
+        N = w.N
+        per_level = []
+        for k in range(w.iters):
+            a, b = tr["ptr"][k * N], tr["ptr"][(k + 1) * N]
+            per_level.append((np.ascontiguousarray(tr["op"][k]), (tr["ptr"][k * N:(k + 1) * N + 1] - a).astype(np.int64),
+                              np.ascontiguousarray(tr["nbr"][a:b]), np.ascontiguousarray(tr["ver"][a:b]),
+                              np.ascontiguousarray(tr["num"][a:b]), np.ascontiguousarray(tr["den"][k])))
+        probe = np.zeros(PROBE, np.float32)
+        n_e2e = min(args.steps, w.iters)
+        for k in range(min(3, w.iters)):
+            h.step_host(*per_level[k], probe)
+        reset()
+        barrier()
+        t0 = time.perf_counter()
+        wi2 = 0
+        for k in range(n_e2e):
+            h.step_host(*per_level[k], probe)
+            wi2 += int(wi_per_level[k])
+        torch.cuda.synchronize()
+        t_e2e = time.perf_counter() - t0
+        if dist is not None:
+            t = torch.tensor([t_e2e], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            t_e2e = float(t.item())
+        h2d = float(np.mean([h.level_stats(k)["U"] * 4 + h.level_stats(k)["normal"] * 4 +
+                             (h.level_stats(k)["normal"] + h.level_stats(k)["jump"]) * 32 +
+                             h.level_stats(k)["entries"] * 8 for k in range(n_e2e)]))
+        e2e = {"value": wi2 / t_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 4.0 * min(PROBE, w.P),
+               "steps": n_e2e, "note": "hop_step_host: level records from host memory through a pinned staging buffer, "
+               "probe of worker 0 read back, stream synchronised every step"}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    peak, peak_kind = measured_peaks()
+    mix_launches = tim["spans"][1]
+    ach = tim["mix_bytes"] / (tim["ms_mix"] * 1e-3) / 1e9 if tim["ms_mix"] > 0 else 0.0
+    traffic = NCU_TRAFFIC.get((args.config, P_global))
+    roofline = {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+                "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": "mix_bulk_kernel" if w.P % 4 == 0 else "mix_staged_kernel",
+                "launches": mix_launches, "avg_launch_ms": tim["ms_mix"] / max(1, mix_launches),
+                "alg_bytes_per_launch": tim["mix_bytes"] / max(1, mix_launches),
+                "frac_of_nominal_8TBs": ach / 8000.0,
+                "other_kernels_ms": {"gradient": tim["ms_grad"], "sparse_apply": tim["ms_apply"]}}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"config {args.config}: {w.name}", "N": w.N, "P": P_global, "P_per_gpu": w.P, "s": w.s, "b": w.b,
+                       "levels": w.iters, "trace_passes": args.steps / w.iters, "parallelism": f"column-sharded x{world}",
+                       "l2": "inputs exceed L2 (ring %.1f GB per GPU)" % (X.numel() * 4 / 1e9) if X.numel() * 4 > 3e8 else "ring fits L2: absolute numbers only",
+                       "protocol_sim_ms": sim_ms},
+            "roofline": roofline, "gpu_launches": int(launches), "clocks": sampler.result()}
+    if e2e is not None:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        wf = inputs.make_workload(args.config, P=args.P)
+        v, desc = oracle_sample(wf)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -181,6 +181,14 @@ int hop_read_status(hop_ctx* ctx, int32_t* device_error_word);
  * JUMP records, consumed entries sum_i |C_{i,k}|, tile width chosen, kernel chosen, staged rows,
  * algorithmic bytes of the mix-update kernel. */
 int hop_level_stats(hop_ctx* ctx, int32_t level, int64_t* out);
+/* Per-kernel-class timing (tracing aid).  While enabled, hop_step / hop_step_host bracket each
+ * kernel class with CUDA events on the bound stream.  hop_timing_read synchronises the stream and
+ * returns, since the last read: ms[3] = {gradient kernels, mix-update kernel, sparse apply}, the
+ * number of timed spans of each class, and the algorithmic bytes of the timed mix-update launches
+ * (per level: every distinct consumed slice once + dense gradient once + result once, + momentum
+ * read and write); then it resets the counters. */
+int hop_timing_enable(hop_ctx* ctx, int32_t on);
+int hop_timing_read(hop_ctx* ctx, double* ms, int64_t* spans, int64_t* mix_bytes);
 /* Number of kernels launched by this context so far. */
 int hop_launch_count(hop_ctx* ctx, int64_t* launches);
 

@@ -47,6 +47,12 @@ struct hop_ctx {
     int32_t* d_err = nullptr;
     int sm_count = 0;
     int64_t launches = 0;
+    // optional per-kernel-class timing with CUDA events on the bound stream
+    bool timing = false;
+    std::vector<cudaEvent_t> ev_pool;
+    size_t ev_used = 0;
+    struct Span { size_t a, b; int kind; int64_t bytes; };
+    std::vector<Span> spans;
     std::string err;
 };
 
@@ -117,6 +123,7 @@ extern "C" int hop_destroy(hop_ctx* c) {
     if (c->d_stage) cudaFree(c->d_stage);
     if (c->h_stage) cudaFreeHost(c->h_stage);
     if (c->h_probe) cudaFreeHost(c->h_probe);
+    for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
     delete c;
     return HOP_OK;
 }
@@ -295,15 +302,31 @@ static int check_mode(hop_ctx* c) {
     return HOP_OK;
 }
 
+static int mark(hop_ctx* c, size_t* idx) {
+    if (c->ev_used == c->ev_pool.size()) {
+        cudaEvent_t e;
+        HOP_CUDA(c, cudaEventCreate(&e));
+        c->ev_pool.push_back(e);
+    }
+    *idx = c->ev_used++;
+    HOP_CUDA(c, cudaEventRecord(c->ev_pool[*idx], c->stream));
+    return HOP_OK;
+}
+#define HOP_SPAN_BEGIN() do { if (c->timing) { int r_ = mark(c, &t0); if (r_) return r_; } } while (0)
+#define HOP_SPAN_END(kind, bytes) do { if (c->timing) { int r_ = mark(c, &t1); if (r_) return r_; \
+    c->spans.push_back({t0, t1, (kind), (int64_t)(bytes)}); } } while (0)
+
 // Enqueues the kernels of one level.
 static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv) {
+    size_t t0 = 0, t1 = 0;
     HopLaunchCfg cfg{};
     cfg.X = c->X; cfg.M = c->M; cfg.G = c->G; cfg.P = c->P; cfg.N = c->g.N; cfg.s = c->s;
     cfg.lr = (float)c->lr; cfg.mu = (float)c->momentum; cfg.tile_w = L.tile_w;
     cfg.use_g = c->grad_mode != HOP_GRAD_SVM_CSR;
     cfg.sm_count = c->sm_count; cfg.err_word = c->d_err; cfg.stream = c->stream;
     int e = 0;
-    if (L.nG > 0) {
+    if (L.nG > 0 && c->grad_mode != HOP_GRAD_EXTERNAL) {
+        HOP_SPAN_BEGIN();
         switch (c->grad_mode) {
         case HOP_GRAD_SYNTHETIC:
             e = hop_launch_synth_grad(cfg, lv, c->grad_seed, (float)c->sigma, c->col_offset); c->launches += 1; break;
@@ -314,16 +337,21 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv) {
         default: break;
         }
         if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("gradient kernel launch: ") + cudaGetErrorString((cudaError_t)e));
+        HOP_SPAN_END(0, 0);
     }
     if (L.nA > 0) {
+        HOP_SPAN_BEGIN();
         e = (L.kernel == HOP_MIX_BULK) ? hop_launch_mix_bulk(cfg, lv) : hop_launch_mix_staged(cfg, lv);
         c->launches += 1;
         if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("mix kernel launch: ") + cudaGetErrorString((cudaError_t)e));
+        HOP_SPAN_END(1, L.alg_bytes);
     }
     if (L.nG > 0 && c->grad_mode == HOP_GRAD_SVM_CSR) {
+        HOP_SPAN_BEGIN();
         e = hop_launch_svm_csr_apply(cfg, lv, c->svmRowPtr, c->svmCol, c->svmVal, c->svmR, c->svmB, c->coef);
         c->launches += 1;
         if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("sparse apply launch: ") + cudaGetErrorString((cudaError_t)e));
+        HOP_SPAN_END(2, 0);
     }
     return HOP_OK;
 }
@@ -466,6 +494,31 @@ extern "C" int hop_level_stats(hop_ctx* c, int32_t level, int64_t* out) {
     const HopLevelHost& L = c->levels[level];
     out[0] = L.U; out[1] = L.nG; out[2] = L.nJump; out[3] = L.sumC; out[4] = L.tile_w; out[5] = L.kernel;
     out[6] = L.stage_rows; out[7] = L.alg_bytes;
+    return HOP_OK;
+}
+
+extern "C" int hop_timing_enable(hop_ctx* c, int32_t on) {
+    if (!c) return HOP_E_ARG;
+    c->timing = on != 0;
+    c->spans.clear();
+    c->ev_used = 0;
+    return HOP_OK;
+}
+
+extern "C" int hop_timing_read(hop_ctx* c, double* ms, int64_t* launches, int64_t* mix_bytes) {
+    if (!c || !ms || !launches || !mix_bytes) return HOP_E_ARG;
+    for (int k = 0; k < 3; ++k) { ms[k] = 0.0; launches[k] = 0; }
+    *mix_bytes = 0;
+    if (c->bound) HOP_CUDA(c, cudaStreamSynchronize(c->stream));
+    for (const auto& sp : c->spans) {
+        float t = 0.f;
+        HOP_CUDA(c, cudaEventElapsedTime(&t, c->ev_pool[sp.a], c->ev_pool[sp.b]));
+        ms[sp.kind] += t;
+        launches[sp.kind] += 1;
+        if (sp.kind == 1) *mix_bytes += sp.bytes;
+    }
+    c->spans.clear();
+    c->ev_used = 0;
     return HOP_OK;
 }
 

@@ -49,6 +49,8 @@ SIGNATURES = {
     "hop_step_host": [_p, _p, _p, _p, _p, _p, _p, _p, _i64],
     "hop_read_status": [_p, C.POINTER(_i32)],
     "hop_level_stats": [_p, _i32, _p],
+    "hop_timing_enable": [_p, _i32],
+    "hop_timing_read": [_p, _p, _p, C.POINTER(_i64)],
     "hop_launch_count": [_p, C.POINTER(_i64)],
 }
 for _name, _args in SIGNATURES.items():
@@ -191,6 +193,14 @@ class Hop:
         out = np.zeros(8, np.int64)
         self._chk(lib.hop_level_stats(self.h, level, _ptr(out)))
         return dict(zip(("U", "normal", "jump", "entries", "tile_w", "kernel", "stage_rows", "alg_bytes"), out.tolist()))
+
+    def timing_enable(self, on=True):
+        self._chk(lib.hop_timing_enable(self.h, 1 if on else 0))
+
+    def timing_read(self):
+        ms, n, b = np.zeros(3, np.float64), np.zeros(3, np.int64), _i64()
+        self._chk(lib.hop_timing_read(self.h, _ptr(ms), _ptr(n), C.byref(b)))
+        return dict(ms_grad=ms[0], ms_mix=ms[1], ms_apply=ms[2], spans=n.tolist(), mix_bytes=b.value)
 
     def launch_count(self):
         n = _i64()
