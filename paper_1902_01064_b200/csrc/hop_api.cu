@@ -234,7 +234,9 @@ static int plan_level(hop_ctx* c, HopLevelHost& L) {
     if (kernel == HOP_MIX_AUTO || kernel == HOP_MIX_TENSOR) kernel = (c->P % 4 == 0) ? HOP_MIX_BULK : HOP_MIX_STAGED;
     if (kernel == HOP_MIX_BULK && c->P % 4 != 0) HOP_FAIL(c, HOP_E_UNSUPPORTED, "the bulk-copy mix kernel needs P to be a multiple of 4");
     const int rows = std::max(1, L.stage_rows);
-    const int64_t budget = hop_mix_smem_budget(kernel) / hop_mix_stages(kernel);
+    const int64_t tb = ((int64_t)L.recs.size() * sizeof(HopRecord) + (int64_t)L.ents.size() * sizeof(HopEntry) + 127) / 128 * 128;
+    L.table_smem = (kernel == HOP_MIX_BULK && tb <= hop_mix_table_limit()) ? (int32_t)tb : 0;
+    const int64_t budget = (hop_mix_smem_budget(kernel) - L.table_smem) / hop_mix_stages(kernel);
     int64_t w = budget / ((int64_t)rows * 4);
     const int unit = (c->P % 4 == 0) ? 4 : 1;
     if (w >= 128) w = std::min<int64_t>(1024, w / 128 * 128);
@@ -245,6 +247,7 @@ static int plan_level(hop_ctx* c, HopLevelHost& L) {
     w = std::min<int64_t>(w, Pr);
     L.tile_w = (int32_t)w;
     L.kernel = kernel;
+    for (HopEntry& e : L.ents) e.u *= L.tile_w;     // slice index -> float offset of its row in a staged tile
     // every distinct consumed slice once + gradient once + result once (+ momentum read and write)
     L.alg_bytes = 4 * c->P * ((int64_t)L.U + nG + L.nA + (mom ? 2 * (int64_t)nG : 0));
     return HOP_OK;
@@ -324,6 +327,7 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv) {
     cfg.lr = (float)c->lr; cfg.mu = (float)c->momentum; cfg.tile_w = L.tile_w;
     cfg.use_g = c->grad_mode != HOP_GRAD_SVM_CSR;
     cfg.sm_count = c->sm_count; cfg.err_word = c->d_err; cfg.stream = c->stream;
+    cfg.table_smem = L.table_smem; cfg.n_ents = (int32_t)L.ents.size();
     int e = 0;
     if (L.nG > 0 && c->grad_mode != HOP_GRAD_EXTERNAL) {
         HOP_SPAN_BEGIN();

@@ -26,7 +26,7 @@ struct HopRecord {          // one active (NORMAL or JUMP) worker of a level
     int32_t pad0, pad1;
 };
 struct HopEntry {
-    int32_t u;              // index into the level's distinct-slice list
+    int32_t u;              // float offset of the slice's row inside a staged tile: slice index * tile width
     float w;                // float(num) / float(den)
 };
 
@@ -40,7 +40,7 @@ struct HopLevelHost {
     // offsets into the uploaded arrays
     int64_t off_src = 0, off_rec = 0, off_ent = 0, off_gw = 0;
     // launch plan
-    int32_t tile_w = 0, kernel = 0, stage_rows = 0;
+    int32_t tile_w = 0, kernel = 0, stage_rows = 0, table_smem = 0;
     int64_t alg_bytes = 0;
 };
 
@@ -85,6 +85,8 @@ struct HopLaunchCfg {
     int32_t use_g;      // dense gradient rows are applied
     int32_t sm_count;
     int32_t* err_word;  // device
+    int32_t table_smem; // bytes of shared memory holding the level's records + entries (0 = read from global)
+    int32_t n_ents;
     void* stream;
 };
 int hop_launch_mix_staged(const HopLaunchCfg& c, const HopLevelDev& lv);
@@ -98,3 +100,4 @@ int hop_launch_svm_csr_apply(const HopLaunchCfg& c, const HopLevelDev& lv, const
                              const float* val, int32_t R, int32_t B, const float* coef);
 int hop_mix_smem_budget(int kernel);   // usable dynamic shared memory per CTA for the kernel
 int hop_mix_stages(int kernel);
+int hop_mix_table_limit();

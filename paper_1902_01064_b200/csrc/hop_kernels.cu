@@ -10,6 +10,7 @@
 // brings every distinct consumed slice of the tile into shared memory, then writes.  Blocks own
 // disjoint columns, so no other ordering is needed, and every distinct slice is read once.
 #include <cuda_runtime.h>
+#include <algorithm>
 #include <cstdint>
 
 #include "hop_internal.h"
@@ -17,8 +18,9 @@
 namespace {
 
 constexpr int kStagedThreads = 256;
-constexpr int kConsumerWarps = 8;
-constexpr int kBulkThreads = 32 * (kConsumerWarps + 1);
+constexpr int kConsumerWarps = 16;
+constexpr int kProducerWarps = 4;   // one warp cannot issue ~200 small bulk copies per tile fast enough (measured)
+constexpr int kBulkThreads = 32 * (kConsumerWarps + kProducerWarps);
 constexpr int kBulkStages = 2;
 constexpr uint32_t kSpinLimit = 1u << 22;
 
@@ -33,6 +35,7 @@ __device__ __forceinline__ void reduce_apply_record(const HopRecord& r, const Ho
                                                     bool use_g, float lr, float mu, float* __restrict__ X,
                                                     float* __restrict__ M, int64_t P, int64_t c0, int lane) {
     const HopEntry* e = ents + r.ent_begin;
+    const int n = r.ent_count;
     float* out = X + (int64_t)r.out_row * P + c0;
     const bool grad = use_g && r.g_stage >= 0;
     const float* grow = stage + (int64_t)(U + (grad ? r.g_stage : 0)) * w;
@@ -41,12 +44,23 @@ __device__ __forceinline__ void reduce_apply_record(const HopRecord& r, const Ho
     for (int c = lane * VEC; c < wd; c += 32 * VEC) {
         if constexpr (VEC == 4) {
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int t = 0; t < r.ent_count; ++t) {
-                const HopEntry en = e[t];
-                const float4 v = *reinterpret_cast<const float4*>(stage + (int64_t)en.u * w + c);
-                acc.x = fmaf(en.w, v.x, acc.x); acc.y = fmaf(en.w, v.y, acc.y);
-                acc.z = fmaf(en.w, v.z, acc.z); acc.w = fmaf(en.w, v.w, acc.w);
+            const float* sc = stage + c;
+            int t = 0;
+#define HOP_FMA4(W, V) acc.x = fmaf(W, V.x, acc.x); acc.y = fmaf(W, V.y, acc.y); acc.z = fmaf(W, V.z, acc.z); acc.w = fmaf(W, V.w, acc.w)
+            for (; t + 4 <= n; t += 4) {      // loads first, then the multiply-adds in entry order
+                const HopEntry e0 = e[t], e1 = e[t + 1], e2 = e[t + 2], e3 = e[t + 3];
+                const float4 v0 = *reinterpret_cast<const float4*>(sc + e0.u);
+                const float4 v1 = *reinterpret_cast<const float4*>(sc + e1.u);
+                const float4 v2 = *reinterpret_cast<const float4*>(sc + e2.u);
+                const float4 v3 = *reinterpret_cast<const float4*>(sc + e3.u);
+                HOP_FMA4(e0.w, v0); HOP_FMA4(e1.w, v1); HOP_FMA4(e2.w, v2); HOP_FMA4(e3.w, v3);
             }
+            for (; t < n; ++t) {
+                const HopEntry en = e[t];
+                const float4 v = *reinterpret_cast<const float4*>(sc + en.u);
+                HOP_FMA4(en.w, v);
+            }
+#undef HOP_FMA4
             if (grad) {
                 float4 g = *reinterpret_cast<const float4*>(grow + c);
                 if constexpr (MOMENTUM) {
@@ -61,9 +75,9 @@ __device__ __forceinline__ void reduce_apply_record(const HopRecord& r, const Ho
             *reinterpret_cast<float4*>(out + c) = acc;
         } else {
             float acc = 0.f;
-            for (int t = 0; t < r.ent_count; ++t) {
+            for (int t = 0; t < n; ++t) {
                 const HopEntry en = e[t];
-                acc = fmaf(en.w, stage[(int64_t)en.u * w + c], acc);
+                acc = fmaf(en.w, stage[en.u + c], acc);
             }
             if (grad) {
                 float g = grow[c];
@@ -143,30 +157,45 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
-// mix_bulk: persistent blocks; warp 0 is the producer (asynchronous bulk copies of every staged row of
-// the next tile, completion counted in bytes on an mbarrier), warps 1..8 consume.  Two stages.
+// mix_bulk: persistent blocks; the first kProducerWarps warps are producers (asynchronous bulk copies of
+// every staged row of the next tile, rows dealt round-robin to the producer lanes, completion counted
+// in bytes on an mbarrier), the other kConsumerWarps warps consume.  Two stages.
 // Requires P % 4 == 0 and 16-byte aligned base pointers (bulk copies move multiples of 16 bytes).
 template <bool MOMENTUM>
 __global__ void __launch_bounds__(kBulkThreads, 1)
 mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __restrict__ G, int64_t P, int w,
-                int use_g, float lr, float mu, HopLevelDev lv, int32_t* __restrict__ err_word) {
+                int use_g, float lr, float mu, HopLevelDev lv, int table_bytes, int n_ents,
+                int32_t* __restrict__ err_word) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw);
     uint64_t* empty = full + kBulkStages;
-    float* stage0 = reinterpret_cast<float*>(smem_raw + 128);
+    float* stage0 = reinterpret_cast<float*>(smem_raw + 128 + table_bytes);
+    // the level's records and entries are read once per tile by every consumer warp: keep them on chip
+    const HopRecord* recs = lv.recs;
+    const HopEntry* ents = lv.ents;
+    if (table_bytes > 0) {
+        HopRecord* srec = reinterpret_cast<HopRecord*>(smem_raw + 128);
+        HopEntry* sent = reinterpret_cast<HopEntry*>(srec + lv.nA);
+        const int4* gr = reinterpret_cast<const int4*>(lv.recs);
+        for (int i = threadIdx.x; i < lv.nA * 2; i += blockDim.x) reinterpret_cast<int4*>(srec)[i] = gr[i];
+        for (int i = threadIdx.x; i < n_ents; i += blockDim.x) sent[i] = lv.ents[i];
+        recs = srec; ents = sent;
+    }
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nG = use_g ? lv.nG : 0;
     const int rows = lv.U + nG * (MOMENTUM ? 2 : 1);
     const int64_t stage_floats = (int64_t)rows * w;
     const int64_t tiles = (P + w - 1) / w;
     if (tid == 0) {
-        for (int s = 0; s < kBulkStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kConsumerWarps); }
+        for (int s = 0; s < kBulkStages; ++s) { mbar_init(&full[s], kProducerWarps); mbar_init(&empty[s], kConsumerWarps); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
-    if (warp == 0) {
-        // ---------------- producer
+    if (warp < kProducerWarps) {
+        // ---------------- producers: this warp issues rows warp*32 + lane, + 32*kProducerWarps, ...
+        int my_rows = 0;
+        for (int r0 = warp * 32; r0 < rows; r0 += 32 * kProducerWarps) my_rows += min(32, rows - r0);
         int64_t n = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++n) {
@@ -176,10 +205,10 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
             const int64_t c0 = tile * w;
             const int wd = (int)min((int64_t)w, P - c0);
             const uint32_t bytes = (uint32_t)wd * 4u;
-            if (lane == 0) mbar_expect_tx(&full[s], bytes * (uint32_t)rows);
+            if (lane == 0) mbar_expect_tx(&full[s], bytes * (uint32_t)my_rows);
             __syncwarp();
             float* dst = stage0 + s * stage_floats;
-            for (int r = lane; r < rows; r += 32) {
+            for (int r = warp * 32 + lane; r < rows; r += 32 * kProducerWarps) {
                 const float* src;
                 if (r < lv.U) src = X + (int64_t)lv.src_row[r] * P;
                 else if (r < lv.U + nG) src = G + (int64_t)lv.grad_workers[r - lv.U] * P;
@@ -195,7 +224,7 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
         }
     } else {
         // ---------------- consumers
-        const int cw = warp - 1;
+        const int cw = warp - kProducerWarps;
         int64_t n = 0;
         for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++n) {
             const int s = (int)(n % kBulkStages);
@@ -205,7 +234,7 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
             const int wd = (int)min((int64_t)w, P - c0);
             const float* st = stage0 + s * stage_floats;
             for (int a = cw; a < lv.nA; a += kConsumerWarps)
-                reduce_apply_record<4, MOMENTUM>(lv.recs[a], lv.ents, st, w, wd, lv.U, nG, use_g != 0, lr, mu, X, M, P, c0, lane);
+                reduce_apply_record<4, MOMENTUM>(recs[a], ents, st, w, wd, lv.U, nG, use_g != 0, lr, mu, X, M, P, c0, lane);
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[s]);
         }
@@ -226,14 +255,17 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
     }
     o[0] = c0; o[1] = c1; o[2] = c2; o[3] = c3;
 }
-// Box-Muller on 23-bit uniforms u = (n + 1/2) / 2^23 (exact in float32).
+// Box-Muller on 23-bit uniforms u = (n + 1/2) / 2^23 (exact in float32).  The hardware approximations
+// __logf / __sincosf are used on purpose: their error (<= 3 ulp for the logarithm, <= 2^-21.4 absolute
+// for sine and cosine on [-pi, pi]) changes a normal deviate by < 3e-6, i.e. a parameter by < 1e-9
+// per step after scaling by sigma and the learning rate, and the kernel is arithmetic-bound otherwise.
 __device__ __forceinline__ void box_muller(uint32_t ra, uint32_t rb, float& z0, float& z1) {
-    const float u1 = (float)(((ra >> 9) << 1) | 1u) * 5.9604644775390625e-08f;   // (2n+1) * 2^-24
-    const float two_u2 = (float)(((rb >> 9) << 1) | 1u) * 1.1920928955078125e-07f;  // 2 * u2
-    const float rad = sqrtf(-2.0f * logf(u1));
+    const float u1 = (float)(((ra >> 9) << 1) | 1u) * 5.9604644775390625e-08f;      // (2n+1) * 2^-24
+    const float two_u2 = (float)(((rb >> 9) << 1) | 1u) * 1.1920928955078125e-07f;  // 2 * u2 in (0, 2)
+    const float rad = sqrtf(-2.0f * __logf(u1));
     float sn, cs;
-    sincospif(two_u2, &sn, &cs);
-    z0 = rad * cs; z1 = rad * sn;
+    __sincosf((two_u2 - 1.0f) * 3.14159265358979323846f, &sn, &cs);                  // angle - pi in (-pi, pi)
+    z0 = -rad * cs; z1 = -rad * sn;                                                  // cos(a) = -cos(a - pi)
 }
 
 __global__ void __launch_bounds__(256)
@@ -344,6 +376,7 @@ size_t staged_smem(const HopLaunchCfg& c, const HopLevelDev& lv) {
 }  // namespace
 
 int hop_mix_smem_budget(int kernel) { return kernel == HOP_MIX_BULK ? (227 * 1024 - 128) : 100 * 1024; }
+int hop_mix_table_limit() { return 32 * 1024; }
 int hop_mix_stages(int kernel) { return kernel == HOP_MIX_BULK ? kBulkStages : 1; }
 
 int hop_launch_mix_staged(const HopLaunchCfg& c, const HopLevelDev& lv) {
@@ -375,7 +408,7 @@ int hop_launch_mix_bulk(const HopLaunchCfg& c, const HopLevelDev& lv) {
     if (lv.nA == 0) return 0;
     const int nG = c.use_g ? lv.nG : 0;
     const int rows = lv.U + nG * (c.mu != 0.f ? 2 : 1);
-    const size_t smem = 128 + (size_t)kBulkStages * rows * c.tile_w * sizeof(float);
+    const size_t smem = 128 + (size_t)c.table_smem + (size_t)kBulkStages * rows * c.tile_w * sizeof(float);
     const int64_t tiles = (c.P + c.tile_w - 1) / c.tile_w;
     const int grid = (int)std::min<int64_t>(tiles, (int64_t)c.sm_count);
     cudaStream_t st = (cudaStream_t)c.stream;
@@ -383,11 +416,11 @@ int hop_launch_mix_bulk(const HopLaunchCfg& c, const HopLevelDev& lv) {
     if (c.mu != 0.f) {
         e = cudaFuncSetAttribute(mix_bulk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return (int)e;
-        mix_bulk_kernel<true><<<grid, kBulkThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, lv, c.err_word);
+        mix_bulk_kernel<true><<<grid, kBulkThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, lv, c.table_smem, c.n_ents, c.err_word);
     } else {
         e = cudaFuncSetAttribute(mix_bulk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return (int)e;
-        mix_bulk_kernel<false><<<grid, kBulkThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, lv, c.err_word);
+        mix_bulk_kernel<false><<<grid, kBulkThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, lv, c.table_smem, c.n_ents, c.err_word);
     }
     return (int)cudaGetLastError();
 }
