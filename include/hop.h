@@ -192,6 +192,35 @@ int hop_timing_read(hop_ctx* ctx, double* ms, int64_t* spans, int64_t* mix_bytes
 /* Number of kernels launched by this context so far. */
 int hop_launch_count(hop_ctx* ctx, int64_t* launches);
 
+/* ---- allocation-free entry point (the paper has no counterpart) -------------------------------
+ * For callers that are not allowed to allocate device memory while they run: code inside a
+ * region where cudaMalloc is forbidden or would synchronise the device (a latency-critical loop,
+ * a plugin hosted by a framework that owns the allocator, a process whose memory budget is fixed
+ * at start-up).  It performs the hinge-loss SVM minibatch step of hop_bind_svm_csr + hop_step for
+ * ONE parameter vector without any context: coef_r = -y_r/rows if y_r * (a_r . x) < 1 else 0,
+ * then x_out[col] -= lr * coef_r * val for every stored element of the `rows` CSR rows.  x_out may
+ * alias x when no mixing happens in between, or hold the mixed parameters.
+ *
+ * The per-row coefficients, which hop_step keeps in a cudaMalloc'ed buffer, are written to a
+ * fixed array of HOP_STATIC_MAX_ROWS floats (64 KiB) inside the library image; every GPU that
+ * loads the library carries it until the process exits.  The call makes no cudaMalloc / cudaFree
+ * and calls no allocating library routine.  rows > HOP_STATIC_MAX_ROWS is rejected with
+ * HOP_E_ARG and a message in errbuf.
+ *
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call outside any stream capture.  All calls on a device share the
+ * array and it keeps the previous call's coefficients (each call overwrites the rows it uses
+ * before reading them, so nothing needs clearing); two calls whose kernels overlap on the GPU
+ * (different streams) race on it -- serialise them.
+ *
+ * x, x_out: device float[P]; row_ptr: device int64[rows+1] offsets into col/val; col: device
+ * int32 (each < P, not checked); val: device float; y: device float[rows] (+1/-1).  Asynchronous
+ * on cuda_stream.  errbuf (host, may be NULL) receives a NUL-terminated message on failure. */
+#define HOP_STATIC_MAX_ROWS 16384
+int hop_svm_csr_sgd_static(const float* x, float* x_out, int64_t P, const int64_t* row_ptr,
+                           const int32_t* col, const float* val, const float* y, int32_t rows,
+                           float lr, void* cuda_stream, char* errbuf, int64_t errbuf_len);
+
 #ifdef __cplusplus
 }
 #endif

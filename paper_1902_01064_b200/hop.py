@@ -52,6 +52,7 @@ SIGNATURES = {
     "hop_timing_enable": [_p, _i32],
     "hop_timing_read": [_p, _p, _p, C.POINTER(_i64)],
     "hop_launch_count": [_p, C.POINTER(_i64)],
+    "hop_svm_csr_sgd_static": [_p, _p, _i64, _p, _p, _p, _p, _i32, C.c_float, _p, C.c_char_p, _i64],
 }
 for _name, _args in SIGNATURES.items():
     _f = getattr(lib, _name)
@@ -214,6 +215,19 @@ class Hop:
 
     def __del__(self):
         self.close()
+
+
+STATIC_MAX_ROWS = 16384
+
+
+def svm_csr_sgd_static(x, x_out, P, row_ptr, col, val, y, rows, lr, stream=None):
+    """hop_svm_csr_sgd_static: context-free hinge-SVM minibatch step that allocates nothing (its
+    coefficient scratch is a fixed array inside the library).  All array arguments are device buffers."""
+    buf = C.create_string_buffer(512)
+    rc = lib.hop_svm_csr_sgd_static(_ptr(x), _ptr(x_out), P, _ptr(row_ptr), _ptr(col), _ptr(val), _ptr(y), rows,
+                                    float(lr), stream, buf, len(buf))
+    if rc:
+        raise HopError(rc, buf.value.decode())
 
 
 def from_workload(w, mix_kernel=MIX_AUTO) -> Hop:
