@@ -278,3 +278,23 @@ def test_malformed_traces_are_rejected_on_the_host():
     load(lambda t: t["op"].__setitem__((2, 0), 7))                            # unknown op
     g.h.load_trace(g.trace)
     g.h.close()
+
+
+def test_column_shards_equal_the_full_run_bitwise():
+    # what `bench.py --gpus N` does per rank: a contiguous column range with HOP_OPT_COL_OFFSET
+    import bench
+    P = 5120
+    w = inputs.make_workload(4, P=P, iters=20)
+    full = GpuRun(w).run(w.iters)
+    for world in (2, 3):
+        for r in range(world):
+            lo, hi = bench.shard_columns(P, world, r)
+            ws = inputs.make_workload(4, P=P, iters=20)
+            p0 = ws.p0()[lo:hi].copy()
+            ws.P, ws._p0 = hi - lo, p0
+            g = GpuRun(ws)
+            g.h.set_option(hop.OPT_COL_OFFSET, lo)
+            got = g.run(ws.iters)
+            for i in range(w.N):
+                assert np.array_equal(got[i], full[i][lo:hi])
+            g.h.close()

@@ -1,0 +1,70 @@
+"""Multi-rank host logic of the column-sharded run (world size 2, gloo, CPU): shard boundaries, the
+max-over-ranks timing reduction, and the fact that the path is separable by column, so that ranks
+working on their own column ranges with the replicated trace reproduce the unsharded result."""
+import os
+import socket
+import sys
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import bench
+from oracle import protocol as op, update as up
+from paper_1902_01064_b200 import inputs
+
+
+def test_shard_columns_partition():
+    for P in (1, 4, 127, 128, 129, 1000, 25_600_000, 8_000_000, 1_200_000):
+        for n in (1, 2, 3, 4, 8):
+            spans = [bench.shard_columns(P, n, r) for r in range(n)]
+            assert spans[0][0] == 0 and spans[-1][1] == P
+            for (a, b), (c, d) in zip(spans, spans[1:]):
+                assert b == c and a <= b
+            assert all(a % 128 == 0 for a, _ in spans)
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def _rank_main(rank, world, port, P, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    w = inputs.make_workload(3, P=P, iters=12)
+    lo, hi = bench.shard_columns(P, world, rank)
+    tr = op.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode).to_arrays()   # replicated
+    cols = np.arange(lo, hi)
+    x0 = np.tile(w.p0()[cols].astype(np.float64), (w.N, 1))
+    X, newest = up.run_updates(tr, w.N, w.lr, w.momentum, x0, up.GradSynthetic(w.grad_seed, w.sigma, cols), s=w.s)
+    mine = np.stack([X[(i, newest[i])] for i in range(w.N)])
+    # the timing reduction bench.py uses: max over ranks
+    t = torch.tensor([10.0 + rank], dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    parts = [None] * world
+    dist.all_gather_object(parts, (lo, hi, mine))
+    dist.barrier()
+    if rank == 0:
+        full = np.concatenate([p[2] for p in sorted(parts, key=lambda p: p[0])], axis=1)
+        np.save(out, full)
+        assert float(t.item()) == 10.0 + world - 1
+    dist.destroy_process_group()
+
+
+def test_two_ranks_reproduce_the_unsharded_run(tmp_path):
+    P = 1000
+    out = str(tmp_path / "sharded.npy")
+    mp.spawn(_rank_main, args=(2, _free_port(), P, out), nprocs=2, join=True)
+    got = np.load(out)
+    w = inputs.make_workload(3, P=P, iters=12)
+    tr = op.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode).to_arrays()
+    x0 = np.tile(w.p0().astype(np.float64), (w.N, 1))
+    X, newest = up.run_updates(tr, w.N, w.lr, w.momentum, x0, up.GradSynthetic(w.grad_seed, w.sigma, np.arange(P)), s=w.s)
+    want = np.stack([X[(i, newest[i])] for i in range(w.N)])
+    assert np.array_equal(got, want)
