@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhop_b200.so")
-SOURCES = ["hop_api.cu", "hop_kernels.cu", "hop_static.cu", "hop_sim.cpp", "hop_trace.cpp"]
+SOURCES = ["hop_api.cu", "hop_kernels.cu", "hop_dense_tc.cu", "hop_static.cu", "hop_sim.cpp", "hop_trace.cpp"]
 
 
 def _nvcc() -> str:

@@ -33,6 +33,9 @@ struct hop_ctx {
     float* coef = nullptr;
     // loaded trace (owned device tables)
     std::vector<HopLevelHost> levels;
+    float* d_tcw = nullptr;         // tensor-core path: weight numerators, row tables, padded slice rows
+    HopTcRow* d_tcrows = nullptr;
+    int32_t* d_tcsrc = nullptr;
     int32_t* d_i32 = nullptr;       // src_row and grad_workers of all levels
     HopRecord* d_rec = nullptr;
     HopEntry* d_ent = nullptr;
@@ -110,7 +113,11 @@ static void free_trace_tables(hop_ctx* c) {
     if (c->d_i32) cudaFree(c->d_i32);
     if (c->d_rec) cudaFree(c->d_rec);
     if (c->d_ent) cudaFree(c->d_ent);
+    if (c->d_tcw) cudaFree(c->d_tcw);
+    if (c->d_tcrows) cudaFree(c->d_tcrows);
+    if (c->d_tcsrc) cudaFree(c->d_tcsrc);
     c->d_i32 = nullptr; c->d_rec = nullptr; c->d_ent = nullptr;
+    c->d_tcw = nullptr; c->d_tcrows = nullptr; c->d_tcsrc = nullptr;
     c->levels.clear();
     c->loaded = false;
 }
@@ -225,12 +232,38 @@ extern "C" int hop_bind_svm_csr(hop_ctx* c, const int64_t* row_ptr, const int32_
 }
 
 // Tile width and kernel for one level: as many columns per tile as the staged rows leave room for.
-static int plan_level(hop_ctx* c, HopLevelHost& L) {
+static int plan_level(hop_ctx* c, HopLevelHost& L, bool allow_tensor = true) {
     const bool use_g = c->grad_mode != HOP_GRAD_SVM_CSR;
     const bool mom = c->momentum != 0.0;
     const int nG = use_g ? L.nG : 0;
     L.stage_rows = L.U + nG * (mom ? 2 : 1);
     int kernel = c->mix_kernel;
+    // Tensor-core path: dense levels only (a contraction over <= 256 distinct slices for <= 128 workers).
+    const bool tc_ok = allow_tensor && c->g.N <= 128 && L.U <= 256 && L.nA > 0 && c->P % 128 == 0 && !mom && (use_g || L.nG == 0) &&
+                       hop_dense_tc_smem((L.U + 31) / 32 * 32) <= (size_t)227 * 1024;
+    const bool dense = L.nA >= 32 && L.sumC >= 32 * (int64_t)L.nA;
+    if (tc_ok && (kernel == HOP_MIX_TENSOR || (kernel == HOP_MIX_AUTO && dense))) {
+        L.kernel = HOP_MIX_TENSOR;
+        L.tile_w = 128;
+        L.stage_rows = L.U;
+        L.Kpad = (L.U + 31) / 32 * 32;
+        L.tc_w.assign((size_t)L.Kpad * 128, 0.f);
+        L.tc_rows.assign(128, HopTcRow{-1, -1, 1.f});
+        L.tc_src.assign(L.Kpad, L.src_row[0]);
+        std::copy(L.src_row.begin(), L.src_row.end(), L.tc_src.begin());
+        for (size_t a = 0; a < L.recs.size(); ++a) {
+            const HopRecord& r = L.recs[a];
+            const int i = r.worker;
+            L.tc_rows[i] = HopTcRow{r.out_row, (r.g_stage >= 0 && use_g) ? i : -1, (float)L.rec_den[a]};
+            for (int t = r.ent_begin; t < r.ent_begin + r.ent_count; ++t) {
+                const int u = L.ent_slice[t];
+                // A^T in the K-major core-matrix layout the MMA reads: [u/4][i/8][i%8][u%4]
+                L.tc_w[(size_t)(u / 4) * 512 + (i / 8) * 32 + (i % 8) * 4 + (u % 4)] = (float)L.ent_num[t];
+            }
+        }
+        L.alg_bytes = 4 * c->P * ((int64_t)L.U + nG + L.nA);
+        return HOP_OK;
+    }
     if (kernel == HOP_MIX_AUTO || kernel == HOP_MIX_TENSOR) kernel = (c->P % 4 == 0) ? HOP_MIX_BULK : HOP_MIX_STAGED;
     if (kernel == HOP_MIX_BULK && c->P % 4 != 0) HOP_FAIL(c, HOP_E_UNSUPPORTED, "the bulk-copy mix kernel needs P to be a multiple of 4");
     const int rows = std::max(1, L.stage_rows);
@@ -273,7 +306,14 @@ extern "C" int hop_load_trace(hop_ctx* c, const hop_trace* t) {
         if (rc2) return rc2;
     }
     std::vector<int32_t> h_i32; std::vector<HopRecord> h_rec; std::vector<HopEntry> h_ent;
+    std::vector<float> h_tcw; std::vector<HopTcRow> h_tcrows; std::vector<int32_t> h_tcsrc;
     for (auto& Lv : levels) {
+        if (Lv.kernel == HOP_MIX_TENSOR) {
+            Lv.off_tcw = (int64_t)h_tcw.size(); h_tcw.insert(h_tcw.end(), Lv.tc_w.begin(), Lv.tc_w.end());
+            Lv.off_tcrows = (int64_t)h_tcrows.size(); h_tcrows.insert(h_tcrows.end(), Lv.tc_rows.begin(), Lv.tc_rows.end());
+            Lv.off_tcsrc = (int64_t)h_tcsrc.size(); h_tcsrc.insert(h_tcsrc.end(), Lv.tc_src.begin(), Lv.tc_src.end());
+            Lv.tc_w.clear(); Lv.tc_w.shrink_to_fit();
+        }
         Lv.off_src = (int64_t)h_i32.size(); h_i32.insert(h_i32.end(), Lv.src_row.begin(), Lv.src_row.end());
         Lv.off_gw = (int64_t)h_i32.size(); h_i32.insert(h_i32.end(), Lv.grad_workers.begin(), Lv.grad_workers.end());
         Lv.off_rec = (int64_t)h_rec.size(); h_rec.insert(h_rec.end(), Lv.recs.begin(), Lv.recs.end());
@@ -286,6 +326,14 @@ extern "C" int hop_load_trace(hop_ctx* c, const hop_trace* t) {
     HOP_CUDA(c, cudaMemcpyAsync(c->d_i32, h_i32.data(), h_i32.size() * sizeof(int32_t), cudaMemcpyHostToDevice, c->stream));
     HOP_CUDA(c, cudaMemcpyAsync(c->d_rec, h_rec.data(), h_rec.size() * sizeof(HopRecord), cudaMemcpyHostToDevice, c->stream));
     HOP_CUDA(c, cudaMemcpyAsync(c->d_ent, h_ent.data(), h_ent.size() * sizeof(HopEntry), cudaMemcpyHostToDevice, c->stream));
+    if (!h_tcw.empty()) {
+        HOP_CUDA(c, cudaMalloc(&c->d_tcw, h_tcw.size() * sizeof(float)));
+        HOP_CUDA(c, cudaMalloc(&c->d_tcrows, h_tcrows.size() * sizeof(HopTcRow)));
+        HOP_CUDA(c, cudaMalloc(&c->d_tcsrc, h_tcsrc.size() * sizeof(int32_t)));
+        HOP_CUDA(c, cudaMemcpyAsync(c->d_tcw, h_tcw.data(), h_tcw.size() * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+        HOP_CUDA(c, cudaMemcpyAsync(c->d_tcrows, h_tcrows.data(), h_tcrows.size() * sizeof(HopTcRow), cudaMemcpyHostToDevice, c->stream));
+        HOP_CUDA(c, cudaMemcpyAsync(c->d_tcsrc, h_tcsrc.data(), h_tcsrc.size() * sizeof(int32_t), cudaMemcpyHostToDevice, c->stream));
+    }
     HOP_CUDA(c, cudaStreamSynchronize(c->stream));   // the host vectors go out of scope
     c->levels = std::move(levels);
     c->sent = std::move(sent);
@@ -345,7 +393,10 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv) {
     }
     if (L.nA > 0) {
         HOP_SPAN_BEGIN();
-        e = (L.kernel == HOP_MIX_BULK) ? hop_launch_mix_bulk(cfg, lv) : hop_launch_mix_staged(cfg, lv);
+        if (L.kernel == HOP_MIX_TENSOR)
+            e = hop_launch_mix_dense_tc(cfg, c->d_tcw + L.off_tcw, c->d_tcrows + L.off_tcrows, c->d_tcsrc + L.off_tcsrc, L.Kpad);
+        else
+            e = (L.kernel == HOP_MIX_BULK) ? hop_launch_mix_bulk(cfg, lv) : hop_launch_mix_staged(cfg, lv);
         c->launches += 1;
         if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("mix kernel launch: ") + cudaGetErrorString((cudaError_t)e));
         HOP_SPAN_END(1, L.alg_bytes);
@@ -395,7 +446,7 @@ extern "C" int hop_step_host(hop_ctx* c, const int32_t* op, const int64_t* ptr, 
     if (rc) return rc;
     HopLevelHost L;
     hop_build_level(c->g, c->s, k, op, ptr, nbr, ver, num, den, L);
-    rc = plan_level(c, L);
+    rc = plan_level(c, L, false);   // the streaming path uploads only the general kernels' tables
     if (rc) return rc;
     // pack [src_row | grad_workers | recs | ents] into one pinned buffer, one H2D copy
     const size_t b_src = L.src_row.size() * 4, b_gw = L.grad_workers.size() * 4;

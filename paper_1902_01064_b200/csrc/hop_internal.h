@@ -30,6 +30,12 @@ struct HopEntry {
     float w;                // float(num) / float(den)
 };
 
+struct HopTcRow {           // per worker, for the tensor-core dense path
+    int32_t out_row;        // row of X receiving the result, -1 if the worker is idle in this level
+    int32_t g_row;          // row of G to apply (= worker), -1 for none
+    float den;              // weight denominator (row scaling)
+};
+
 struct HopLevelHost {
     int32_t U = 0, nA = 0, nG = 0, nJump = 0;
     int64_t sumC = 0;
@@ -37,6 +43,13 @@ struct HopLevelHost {
     std::vector<HopRecord> recs;        // [nA]
     std::vector<HopEntry> ents;
     std::vector<int32_t> grad_workers;  // [nG] workers with a NORMAL record
+    std::vector<int32_t> ent_slice, ent_num, rec_den;   // integer view of the entries (slice index, numerator), per-record denominator
+    // tensor-core dense path (only when planned): numerators in the MMA's shared-memory layout, row table, padded slice rows
+    int32_t Kpad = 0;
+    std::vector<float> tc_w;
+    std::vector<HopTcRow> tc_rows;
+    std::vector<int32_t> tc_src;
+    int64_t off_tcw = 0, off_tcrows = 0, off_tcsrc = 0;
     // offsets into the uploaded arrays
     int64_t off_src = 0, off_rec = 0, off_ent = 0, off_gw = 0;
     // launch plan
@@ -101,3 +114,6 @@ int hop_launch_svm_csr_apply(const HopLaunchCfg& c, const HopLevelDev& lv, const
 int hop_mix_smem_budget(int kernel);   // usable dynamic shared memory per CTA for the kernel
 int hop_mix_stages(int kernel);
 int hop_mix_table_limit();
+// hop_dense_tc.cu
+size_t hop_dense_tc_smem(int Kpad);
+int hop_launch_mix_dense_tc(const HopLaunchCfg& c, const float* Wk, const HopTcRow* tbl, const int32_t* src_row, int Kpad);

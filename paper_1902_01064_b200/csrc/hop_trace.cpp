@@ -133,7 +133,10 @@ void hop_build_level(const HopGraph& g, int32_t s, int32_t level, const int32_t*
             const int32_t row = nbr[t] * S + ver[t] % S;
             if (slice_of[row] < 0) { slice_of[row] = out.U++; out.src_row.push_back(row); }
             out.ents.push_back({slice_of[row], (float)num[t] / (float)den[i]});
+            out.ent_slice.push_back(slice_of[row]);
+            out.ent_num.push_back(num[t]);
         }
+        out.rec_den.push_back(den[i]);
         out.sumC += r.ent_count;
         out.recs.push_back(r);
     }

@@ -156,17 +156,33 @@ def test_cfg4_full_size_sampled_columns():
 
 
 # ------------------------------------------------------------------ configuration 5: complete graph, 128 workers
-@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("kernel", KERNELS + [hop.MIX_TENSOR])
 def test_cfg5_reduced_full_run(kernel):
     w = inputs.make_workload(5, P=1536)
+    g = GpuRun(w, kernel)
+    assert g.h.level_stats(3)["kernel"] == kernel                      # the requested kernel is the one that runs
+    g.h.close()
     check(w, w.iters, TOL_RUN, kernel)
     check(w, 1, TOL_STEP, kernel, perturb=True)
+
+
+def test_cfg5_tensor_path_many_tiles_and_consensus_start():
+    # more tiles than thread blocks (pipeline wrap-around, accumulator hand-over), and the workload's own
+    # start where all replicas are equal (largest accumulators, every product of equal sign)
+    w = inputs.make_workload(5, P=128 * 700, iters=6)
+    check(w, 1, TOL_STEP, hop.MIX_TENSOR)
+    check(w, w.iters, TOL_RUN, hop.MIX_TENSOR)
+    check(w, 1, TOL_STEP, hop.MIX_TENSOR, perturb=True)
 
 
 def test_cfg5_full_size_sampled_columns_first_levels():
     w = inputs.make_workload(5)
     cols = np.unique(np.concatenate([np.arange(0, w.P, 40009), [w.P - 1, w.P - 3, 127, 128, 255, 256]]))
+    g = GpuRun(w)
+    assert g.h.level_stats(1)["kernel"] == hop.MIX_TENSOR              # what bench.py --config 5 times
+    g.h.close()
     check(w, 4, TOL_RUN, cols=cols)
+    check(w, 1, TOL_STEP, cols=cols, perturb=True)
 
 
 # ------------------------------------------------------------------ kernels in isolation / edge cases
