@@ -36,6 +36,8 @@ struct hop_ctx {
     float* d_tcw = nullptr;         // tensor-core path: weight numerators, row tables, padded slice rows
     HopTcRow* d_tcrows = nullptr;
     int32_t* d_tcsrc = nullptr;
+    alignas(64) unsigned char tc_mapX[128], tc_mapG[128], tc_mapY[8 * 128];   // TMA tensor maps over X, G, output slots
+    int32_t tc_slots = 0;
     int32_t* d_i32 = nullptr;       // src_row and grad_workers of all levels
     HopRecord* d_rec = nullptr;
     HopEntry* d_ent = nullptr;
@@ -240,7 +242,7 @@ static int plan_level(hop_ctx* c, HopLevelHost& L, bool allow_tensor = true) {
     int kernel = c->mix_kernel;
     // Tensor-core path: dense levels only (a contraction over <= 256 distinct slices for <= 128 workers).
     const bool tc_ok = allow_tensor && c->g.N <= 128 && L.U <= 256 && L.nA > 0 && c->P % 128 == 0 && !mom && (use_g || L.nG == 0) &&
-                       hop_dense_tc_smem((L.U + 31) / 32 * 32) <= (size_t)227 * 1024;
+                       hop_dense_tc_smem((L.U + 31) / 32 * 32) > 0;
     const bool dense = L.nA >= 32 && L.sumC >= 32 * (int64_t)L.nA;
     if (tc_ok && (kernel == HOP_MIX_TENSOR || (kernel == HOP_MIX_AUTO && dense))) {
         L.kernel = HOP_MIX_TENSOR;
@@ -254,7 +256,7 @@ static int plan_level(hop_ctx* c, HopLevelHost& L, bool allow_tensor = true) {
         for (size_t a = 0; a < L.recs.size(); ++a) {
             const HopRecord& r = L.recs[a];
             const int i = r.worker;
-            L.tc_rows[i] = HopTcRow{r.out_row, (r.g_stage >= 0 && use_g) ? i : -1, (float)L.rec_den[a]};
+            L.tc_rows[i] = HopTcRow{r.out_row, (r.g_stage >= 0 && use_g) ? i : -1, 1.0f / (float)L.rec_den[a]};
             for (int t = r.ent_begin; t < r.ent_begin + r.ent_count; ++t) {
                 const int u = L.ent_slice[t];
                 // A^T in the K-major core-matrix layout the MMA reads: [u/4][i/8][i%8][u%4]
@@ -333,6 +335,10 @@ extern "C" int hop_load_trace(hop_ctx* c, const hop_trace* t) {
         HOP_CUDA(c, cudaMemcpyAsync(c->d_tcw, h_tcw.data(), h_tcw.size() * sizeof(float), cudaMemcpyHostToDevice, c->stream));
         HOP_CUDA(c, cudaMemcpyAsync(c->d_tcrows, h_tcrows.data(), h_tcrows.size() * sizeof(HopTcRow), cudaMemcpyHostToDevice, c->stream));
         HOP_CUDA(c, cudaMemcpyAsync(c->d_tcsrc, h_tcsrc.data(), h_tcsrc.size() * sizeof(int32_t), cudaMemcpyHostToDevice, c->stream));
+        c->tc_slots = (c->s + 1 <= 8) ? c->s + 1 : 0;
+        const int me = hop_dense_tc_make_maps(c->X, (int64_t)c->g.N * (c->s + 1), c->G, c->g.N, c->P, c->tc_mapX, c->tc_mapG,
+                                              c->tc_mapY, c->tc_slots);
+        if (me) HOP_FAIL(c, HOP_E_CUDA, std::string("tensor map for the dense path: ") + cudaGetErrorString((cudaError_t)me));
     }
     HOP_CUDA(c, cudaStreamSynchronize(c->stream));   // the host vectors go out of scope
     c->levels = std::move(levels);
@@ -394,7 +400,9 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv) {
     if (L.nA > 0) {
         HOP_SPAN_BEGIN();
         if (L.kernel == HOP_MIX_TENSOR)
-            e = hop_launch_mix_dense_tc(cfg, c->d_tcw + L.off_tcw, c->d_tcrows + L.off_tcrows, c->d_tcsrc + L.off_tcsrc, L.Kpad);
+            e = hop_launch_mix_dense_tc(cfg, c->tc_mapX, c->tc_mapG,
+                                        (L.nA == c->g.N && c->tc_slots > 0) ? c->tc_mapY + 128 * ((lv.level + 1) % (c->s + 1)) : nullptr,
+                                        c->d_tcw + L.off_tcw, c->d_tcrows + L.off_tcrows, c->d_tcsrc + L.off_tcsrc, L.Kpad);
         else
             e = (L.kernel == HOP_MIX_BULK) ? hop_launch_mix_bulk(cfg, lv) : hop_launch_mix_staged(cfg, lv);
         c->launches += 1;

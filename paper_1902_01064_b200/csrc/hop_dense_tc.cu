@@ -11,31 +11,38 @@
 // float32 in the epilogue where the row scaling 1/den_i is applied.
 //
 // Roles inside one persistent thread block (one per SM), tile = 128 parameter columns x all workers:
-//   warp 0      producer: cp.async.bulk of the 32 raw X row pieces of a K-chunk into shared memory
+//   warp 0      producer: the 16 raw X row pieces of a K-chunk, four TMA tile::gather4 loads (4 arbitrary rows of
+//               the ring per instruction; issuing one copy per row would be issue-bound: ~27 ns per copy and lane)
 //   warp 1      MMA issue (one elected lane): tcgen05.mma kind::tf32, M=128 (columns) x N=128 (workers) x K=8,
 //               A operand (X_hi / X_lo) from tensor memory, B operand (A^T, resident) from shared memory
+//   warp 3      gradient producer: one 2-D TMA box load of the tile's N x 128 piece of G into shared memory
 //   warps 4-7   converters: lane = column; read the raw chunk from shared memory, split hi/lo with
 //               cvt.rna.tf32, tcgen05.st into the A stages in tensor memory
-//   warps 8-11  epilogue: tcgen05.ld both accumulators, add, release them, then y = acc/den - lr*g with
-//               coalesced 128-byte loads of G and stores of Y per (warp, worker)
-// Tensor memory (512 columns): D_hi 0..127, D_lo 128..255, four A stages of 64 columns (hi 32 + lo 32).
+//   warps 8-11  epilogue: tcgen05.ld both accumulators, add, release them, then y = acc/den - lr*g written over g
+//               in shared memory; the finished N x 128 tile goes to the output slot as one TMA box store (or
+//               one bulk row copy per active worker when some workers are idle in the level)
+// Tensor memory (512 columns): D_hi 0..127, D_lo 128..255, eight A stages of 32 columns (hi 16 + lo 16).
+// Shared memory: control block, A^T (Kpad x 512 B), the G tile (64 KB), 3..8 raw stages of 8 KB.
 // Every wait is bounded; a time-out sets the error word and lets the block run to its normal exit,
 // where tensor memory is released.
+#include <cuda.h>            // CUtensorMap and the cuTensorMapEncodeTiled prototype only; no libcuda link
 #include <cuda_runtime.h>
 
 #include <algorithm>
 #include <cstdint>
+#include <cstring>
 
 #include "hop_internal.h"
 
 namespace {
 
 constexpr int kTile = 128;          // parameter columns per tile = MMA M
-constexpr int kChunk = 32;          // K rows per pipeline stage
-constexpr int kStages = 4;
+constexpr int kChunk = 16;          // K rows per pipeline stage
+constexpr int kStages = 8;          // tensor-memory A stages; raw shared-memory stages: 3..8, chosen by the host
 constexpr int kThreads = 12 * 32;
 constexpr uint32_t kSpin = 1u << 20;
-constexpr int kRawStageBytes = kChunk * kTile * 4;          // 16 KB
+constexpr int kRawStageBytes = kChunk * kTile * 4;          // 8 KB
+constexpr int kGTileBytes = 128 * kTile * 4;                // 64 KB
 enum : int32_t { ERR_TC_WAIT = 3 << 24 };
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -59,6 +66,15 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(s32(dst)), "l"(src), "r"(bytes), "r"(s32(bar)) : "memory");
 }
+// TMA tensor-map loads (2-D, no swizzle).  x is the column (multiple of 4 floats: 16-byte rule), y the row.
+__device__ __forceinline__ void tma_gather4(void* dst, const CUtensorMap* map, int x, int y0, int y1, int y2, int y3, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+                 ::"r"(s32(dst)), "l"(map), "r"(x), "r"(y0), "r"(y1), "r"(y2), "r"(y3), "r"(s32(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_tile2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(s32(dst)), "l"(map), "r"(x), "r"(y), "r"(s32(bar)) : "memory");
+}
 __device__ __forceinline__ uint32_t to_tf32(float x) { uint32_t r; asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x)); return r; }
 
 // Shared-memory matrix descriptor, K-major, no swizzle: 8x(16 B) core matrices; leading-dimension byte
@@ -81,13 +97,10 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
 __device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
-                 "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
                  ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]),
-                 "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]),
-                 "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]),
-                 "r"(v[30]), "r"(v[31]) : "memory");
+                 "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     uint32_t r[32];
@@ -104,20 +117,24 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 
 struct TcSmem {                       // control block at the start of dynamic shared memory
     uint64_t raw_full[kStages], raw_empty[kStages], a_full[kStages], a_empty[kStages];
-    uint64_t acc_full, acc_empty, w_full;
+    uint64_t acc_full, acc_empty, w_full, g_full, g_empty;
     uint32_t tmem_base;
     int abort_flag;
+    int epi_fail;
     HopTcRow rows[128];
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
-mix_dense_tc_kernel(float* __restrict__ X, const float* __restrict__ G, int64_t P, float lr, const float* __restrict__ Wk,
-                    const HopTcRow* __restrict__ tbl, const int32_t* __restrict__ src_row, int Kpad,
+mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapG,
+                    const __grid_constant__ CUtensorMap mapY, int box_store,
+                    float* __restrict__ X, int64_t P, int n_workers, float lr, const float* __restrict__ Wk,
+                    const HopTcRow* __restrict__ tbl, const int32_t* __restrict__ src_row, int Kpad, int raw_stages,
                     int32_t* __restrict__ err_word) {
     extern __shared__ __align__(1024) unsigned char smem[];
     TcSmem* cb = reinterpret_cast<TcSmem*>(smem);
     float* Wsm = reinterpret_cast<float*>(smem + 4096);                        // Kpad * 512 bytes, canonical K-major
-    float* raw = reinterpret_cast<float*>(smem + 4096 + (size_t)Kpad * 512);   // kStages x [32][128] floats
+    float* Gsm = reinterpret_cast<float*>(smem + 4096 + (size_t)Kpad * 512);   // [128 workers][128 columns]
+    float* raw = Gsm + 128 * kTile;                                            // raw_stages x [16][128] floats
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int64_t tiles = P / kTile;
     const int nchunks = Kpad / kChunk;
@@ -126,7 +143,9 @@ mix_dense_tc_kernel(float* __restrict__ X, const float* __restrict__ G, int64_t 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mb_init(&cb->raw_full[s], 1); mb_init(&cb->raw_empty[s], 4); mb_init(&cb->a_full[s], 4); mb_init(&cb->a_empty[s], 1); }
         mb_init(&cb->acc_full, 1); mb_init(&cb->acc_empty, 4); mb_init(&cb->w_full, 1);
+        mb_init(&cb->g_full, 1); mb_init(&cb->g_empty, 1);
         cb->abort_flag = 0;
+        cb->epi_fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -151,14 +170,16 @@ mix_dense_tc_kernel(float* __restrict__ X, const float* __restrict__ G, int64_t 
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
             for (int c = 0; c < nchunks && ok; ++c, ++q) {
-                const int s = (int)(q % kStages);
-                const uint32_t ph = (uint32_t)((q / kStages) & 1);
+                const int s = (int)(q % raw_stages);
+                const uint32_t ph = (uint32_t)((q / raw_stages) & 1);
                 if (!mb_wait(&cb->raw_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
                 if (lane == 0) mb_expect_tx(&cb->raw_full[s], kRawStageBytes);
                 __syncwarp();
-                const int u = c * kChunk + lane;
-                bulk_g2s(raw + (size_t)s * (kChunk * kTile) + lane * kTile, X + (int64_t)src_row[u] * P + tile * kTile,
-                         kTile * 4u, &cb->raw_full[s]);
+                if (lane < kChunk / 4) {
+                    const int u = c * kChunk + lane * 4;
+                    tma_gather4(raw + (size_t)s * (kChunk * kTile) + lane * 4 * kTile, &mapX, (int)(tile * kTile),
+                                src_row[u], src_row[u + 1], src_row[u + 2], src_row[u + 3], &cb->raw_full[s]);
+                }
             }
         }
         if (!ok && lane == 0) { atomicCAS(err_word, 0, ERR_TC_WAIT | 1); cb->abort_flag = 1; }
@@ -175,7 +196,7 @@ mix_dense_tc_kernel(float* __restrict__ X, const float* __restrict__ G, int64_t 
                     const int s = (int)(q % kStages);
                     if (!mb_wait(&cb->a_full[s], (uint32_t)((q / kStages) & 1), abort_flag)) { ok = false; break; }
                     fence_after();
-                    const uint32_t a_hi = tmem + kA0 + s * 64, a_lo = a_hi + 32;
+                    const uint32_t a_hi = tmem + kA0 + s * 32, a_lo = a_hi + 16;
 #pragma unroll
                     for (int j = 0; j < kChunk / 8; ++j) {
                         // B operand: 8 K-columns of A^T = two core-matrix columns, 2048 bytes apart; 8-row groups 128 bytes apart
@@ -191,6 +212,22 @@ mix_dense_tc_kernel(float* __restrict__ X, const float* __restrict__ G, int64_t 
             }
             if (!ok) { atomicCAS(err_word, 0, ERR_TC_WAIT | 2); cb->abort_flag = 1; }
         }
+    } else if (warp == 3) {
+        // ------------------------------------------------ gradient tile producer
+        int n_rows = 0;
+        for (int i = 0; i < 128; ++i) n_rows += (cb->rows[i].g_row >= 0);
+        int64_t tcount = 0;
+        bool ok = true;
+        if (n_rows > 0)
+            for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++tcount) {
+                if (!mb_wait(&cb->g_empty, (uint32_t)((tcount & 1) ^ 1), abort_flag)) { ok = false; break; }
+                if (lane == 0) {      // rows 0..n_workers-1 of G, columns of this tile, in one box
+                    mb_expect_tx(&cb->g_full, (uint32_t)n_workers * kTile * 4u);
+                    tma_tile2d(Gsm, &mapG, (int)(tile * kTile), 0, &cb->g_full);
+                }
+                __syncwarp();
+            }
+        if (!ok && lane == 0) { atomicCAS(err_word, 0, ERR_TC_WAIT | 5); cb->abort_flag = 1; }
     } else if (warp >= 4 && warp < 8) {
         // ------------------------------------------------ converters (lane quarter = warp % 4)
         const int col = (warp - 4) * 32 + lane;
@@ -199,25 +236,25 @@ mix_dense_tc_kernel(float* __restrict__ X, const float* __restrict__ G, int64_t 
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
             for (int c = 0; c < nchunks; ++c, ++q) {
-                const int s = (int)(q % kStages);
-                const uint32_t ph = (uint32_t)((q / kStages) & 1);
-                if (!mb_wait(&cb->raw_full[s], ph, abort_flag) || !mb_wait(&cb->a_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+                const int s = (int)(q % kStages), rs = (int)(q % raw_stages);
+                if (!mb_wait(&cb->raw_full[rs], (uint32_t)((q / raw_stages) & 1), abort_flag) ||
+                    !mb_wait(&cb->a_empty[s], (uint32_t)(((q / kStages) & 1) ^ 1), abort_flag)) { ok = false; break; }
                 fence_after();
-                const float* r = raw + (size_t)s * (kChunk * kTile) + col;
-                uint32_t hi[32], lo[32];
+                const float* r = raw + (size_t)rs * (kChunk * kTile) + col;
+                uint32_t hi[kChunk], lo[kChunk];
 #pragma unroll
-                for (int u = 0; u < 32; ++u) {
+                for (int u = 0; u < kChunk; ++u) {
                     const float x = r[u * kTile];
                     hi[u] = to_tf32(x);
                     lo[u] = to_tf32(x - __uint_as_float(hi[u]));
                 }
-                const uint32_t a_hi = tmem + lane_base + kA0 + s * 64;
-                tmem_st32(a_hi, hi);
-                tmem_st32(a_hi + 32, lo);
+                const uint32_t a_hi = tmem + lane_base + kA0 + s * 32;
+                tmem_st16(a_hi, hi);
+                tmem_st16(a_hi + 16, lo);
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 fence_before();
                 __syncwarp();
-                if (lane == 0) { mb_arrive(&cb->a_full[s]); mb_arrive(&cb->raw_empty[s]); }
+                if (lane == 0) { mb_arrive(&cb->a_full[s]); mb_arrive(&cb->raw_empty[rs]); }
             }
         }
         if (!ok && lane == 0) { atomicCAS(err_word, 0, ERR_TC_WAIT | 3); cb->abort_flag = 1; }
@@ -225,38 +262,69 @@ mix_dense_tc_kernel(float* __restrict__ X, const float* __restrict__ G, int64_t 
         // ------------------------------------------------ epilogue (lane quarter = warp % 4)
         const int col = (warp - 8) * 32 + lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        bool has_g = false;
+        for (int i = 0; i < 128; ++i) has_g |= (cb->rows[i].g_row >= 0);
         int64_t tcount = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++tcount) {
-            if (!mb_wait(&cb->acc_full, (uint32_t)(tcount & 1), abort_flag)) { ok = false; break; }
-            fence_after();
-            float acc[128];
+            // A warp whose wait times out still walks through both named barriers of the iteration and
+            // raises epi_fail, so that all four epilogue warps leave the loop together.
+            bool fail = !mb_wait(&cb->acc_full, (uint32_t)(tcount & 1), abort_flag);
+            if (!fail) {
+                fence_after();
+                float acc[128];
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                float h[32], l[32];
-                tmem_ld32(tmem + lane_base + kDhi + b * 32, h);
-                tmem_ld32(tmem + lane_base + kDlo + b * 32, l);
+                for (int b = 0; b < 4; ++b) {
+                    float h[32], l[32];
+                    tmem_ld32(tmem + lane_base + kDhi + b * 32, h);
+                    tmem_ld32(tmem + lane_base + kDlo + b * 32, l);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) acc[b * 32 + i] = h[i] + l[i];
-            }
-            fence_before();
-            __syncwarp();
-            if (lane == 0) mb_arrive(&cb->acc_empty);       // the next tile's MMAs may overwrite the accumulators now
-            const int64_t c0 = tile * kTile + col;
-#pragma unroll
-            for (int b = 0; b < 128; b += 16) {
-                float g[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const HopTcRow rw = cb->rows[b + i];
-                    g[i] = (rw.g_row >= 0) ? __ldcs(G + (int64_t)rw.g_row * P + c0) : 0.f;
+                    for (int i = 0; i < 32; ++i) acc[b * 32 + i] = h[i] + l[i];
                 }
+                fence_before();
+                __syncwarp();
+                if (lane == 0) mb_arrive(&cb->acc_empty);   // the next tile's MMAs may overwrite the accumulators now
+                fail = has_g && !mb_wait(&cb->g_full, (uint32_t)(tcount & 1), abort_flag);
+                if (!fail) {
+                    // y = acc/den - lr*g replaces g in the shared tile (column-per-thread: conflict-free), then the
+                    // tile leaves through the copy engine: per-thread 4-byte global stores of 128 different rows
+                    // were the slowest part of the kernel by far (measured)
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const HopTcRow rw = cb->rows[b + i];
-                    if (rw.out_row >= 0) X[(int64_t)rw.out_row * P + c0] = fmaf(-lr, g[i], __fdiv_rn(acc[b + i], rw.den));
+                    for (int i = 0; i < 128; ++i) {
+                        const HopTcRow rw = cb->rows[i];
+                        if (rw.out_row >= 0) {
+                            const float g = (rw.g_row >= 0) ? Gsm[i * kTile + col] : 0.f;
+                            Gsm[i * kTile + col] = fmaf(-lr, g, acc[i] * rw.inv_den);
+                        }
+                    }
                 }
             }
+            if (fail) *((volatile int*)&cb->epi_fail) = 1;
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            const bool any_fail = *((volatile int*)&cb->epi_fail) != 0;
+            if (!any_fail) {
+                if (box_store) {
+                    if (warp == 8 && lane == 0) {  // all workers active: one box [n_workers x 128] into the output slot
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                                     ::"l"(&mapY), "r"((int)(tile * kTile)), "r"(0), "r"(s32(Gsm)) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    }
+                } else {                           // one 512-byte row copy per active worker
+                    const int e = tid - 8 * 32;
+                    const HopTcRow rw = cb->rows[e];
+                    if (rw.out_row >= 0) {
+                        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                                     ::"l"(X + (int64_t)rw.out_row * P + tile * kTile), "r"(s32(Gsm + e * kTile)), "r"(kTile * 4) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    }
+                }
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");   // the tile has been read out of shared memory
+            if (any_fail) { ok = false; break; }
+            if (has_g && warp == 8 && lane == 0) mb_arrive(&cb->g_empty);    // the next tile's gradient rows may land now
         }
         if (!ok && lane == 0) { atomicCAS(err_word, 0, ERR_TC_WAIT | 4); cb->abort_flag = 1; }
     }
@@ -267,14 +335,80 @@ mix_dense_tc_kernel(float* __restrict__ X, const float* __restrict__ G, int64_t 
 
 }  // namespace
 
-size_t hop_dense_tc_smem(int Kpad) { return 4096 + (size_t)Kpad * 512 + (size_t)kStages * kRawStageBytes; }
+static int raw_stages_for(int Kpad) {
+    const long free_bytes = 227L * 1024 - 4096 - (long)Kpad * 512 - kGTileBytes;
+    return (int)std::max(0L, std::min<long>(kStages, free_bytes / kRawStageBytes));
+}
+// 0 when the level does not fit (fewer than 3 raw stages)
+size_t hop_dense_tc_smem(int Kpad) {
+    const int st = raw_stages_for(Kpad);
+    return st < 3 ? 0 : 4096 + (size_t)Kpad * 512 + kGTileBytes + (size_t)st * kRawStageBytes;
+}
 
-int hop_launch_mix_dense_tc(const HopLaunchCfg& c, const float* Wk, const HopTcRow* tbl, const int32_t* src_row, int Kpad) {
+// Tensor maps: X as [N*(s+1) rows][P] with a one-row box of 128 columns (the tile::gather4 form loads four
+// such rows), G as [N rows][P] with an N x 128 box.  cuTensorMapEncodeTiled is looked up through the
+// runtime so that the library does not link against the driver.
+// mapY[slot]: the rows {i*(s+1) + slot} of X, i.e. the output slot of a level, as an [N rows][P] tensor with row
+// stride (s+1)*P and an N x 128 box (n_slots maps of 128 bytes each).
+int hop_dense_tc_make_maps(float* X, int64_t ring_rows, const float* G, int32_t N, int64_t P, void* mapX, void* mapG,
+                           void* mapY, int32_t n_slots) {
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn encode = nullptr;
+    if (!encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+        if (e != cudaSuccess) return (int)e;
+        if (!fn || q != cudaDriverEntryPointSuccess) return (int)cudaErrorNotSupported;
+        encode = (EncodeFn)fn;
+    }
+    alignas(64) CUtensorMap m;
+    const cuuint32_t estr[2] = {1, 1};
+    {
+        const cuuint64_t dims[2] = {(cuuint64_t)P, (cuuint64_t)ring_rows};
+        const cuuint64_t strides[1] = {(cuuint64_t)P * 4};
+        const cuuint32_t box[2] = {(cuuint32_t)kTile, 1};
+        if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, X, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return (int)cudaErrorInvalidValue;
+        std::memcpy(mapX, &m, sizeof(m));
+    }
+    if (G) {
+        const cuuint64_t dims[2] = {(cuuint64_t)P, (cuuint64_t)N};
+        const cuuint64_t strides[1] = {(cuuint64_t)P * 4};
+        const cuuint32_t box[2] = {(cuuint32_t)kTile, (cuuint32_t)N};
+        if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(G), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return (int)cudaErrorInvalidValue;
+    }
+    std::memcpy(mapG, &m, sizeof(m));
+    const int64_t S = ring_rows / N;
+    for (int slot = 0; slot < n_slots; ++slot) {
+        const cuuint64_t dims[2] = {(cuuint64_t)P, (cuuint64_t)N};
+        const cuuint64_t strides[1] = {(cuuint64_t)S * P * 4};
+        const cuuint32_t box[2] = {(cuuint32_t)kTile, (cuuint32_t)N};
+        if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, X + (int64_t)slot * P, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return (int)cudaErrorInvalidValue;
+        std::memcpy((unsigned char*)mapY + 128 * slot, &m, sizeof(m));
+    }
+    return 0;
+}
+
+int hop_launch_mix_dense_tc(const HopLaunchCfg& c, const void* mapX, const void* mapG, const void* mapY, const float* Wk,
+                            const HopTcRow* tbl, const int32_t* src_row, int Kpad) {
+    alignas(64) CUtensorMap mx, mg, my;
+    std::memcpy(&mx, mapX, sizeof(mx));
+    std::memcpy(&mg, mapG, sizeof(mg));
+    std::memcpy(&my, mapY ? mapY : mapX, sizeof(my));
     const size_t smem = hop_dense_tc_smem(Kpad);
     cudaError_t e = cudaFuncSetAttribute(mix_dense_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
     const int64_t tiles = c.P / kTile;
     const int grid = (int)std::min<int64_t>(tiles, (int64_t)c.sm_count);
-    mix_dense_tc_kernel<<<grid, kThreads, smem, (cudaStream_t)c.stream>>>(c.X, c.G, c.P, c.lr, Wk, tbl, src_row, Kpad, c.err_word);
+    mix_dense_tc_kernel<<<grid, kThreads, smem, (cudaStream_t)c.stream>>>(mx, mg, my, mapY ? 1 : 0, c.X, c.P, c.N, c.lr, Wk, tbl, src_row, Kpad,
+                                                                          raw_stages_for(Kpad), c.err_word);
     return (int)cudaGetLastError();
 }

@@ -33,7 +33,7 @@ struct HopEntry {
 struct HopTcRow {           // per worker, for the tensor-core dense path
     int32_t out_row;        // row of X receiving the result, -1 if the worker is idle in this level
     int32_t g_row;          // row of G to apply (= worker), -1 for none
-    float den;              // weight denominator (row scaling)
+    float inv_den;          // 1 / weight denominator (row scaling)
 };
 
 struct HopLevelHost {
@@ -116,4 +116,8 @@ int hop_mix_stages(int kernel);
 int hop_mix_table_limit();
 // hop_dense_tc.cu
 size_t hop_dense_tc_smem(int Kpad);
-int hop_launch_mix_dense_tc(const HopLaunchCfg& c, const float* Wk, const HopTcRow* tbl, const int32_t* src_row, int Kpad);
+int hop_dense_tc_make_maps(float* X, int64_t ring_rows, const float* G, int32_t N, int64_t P, void* mapX, void* mapG,
+                           void* mapY, int32_t n_slots);   // 128-byte blobs; mapY holds n_slots of them
+// mapY = the output slot's map when every worker is active in the level, else nullptr (row-by-row stores)
+int hop_launch_mix_dense_tc(const HopLaunchCfg& c, const void* mapX, const void* mapG, const void* mapY, const float* Wk,
+                            const HopTcRow* tbl, const int32_t* src_row, int Kpad);

@@ -175,6 +175,25 @@ def test_cfg5_tensor_path_many_tiles_and_consensus_start():
     check(w, 1, TOL_STEP, hop.MIX_TENSOR, perturb=True)
 
 
+def test_tensor_path_with_idle_and_jumping_workers_and_fewer_than_128_workers():
+    # not every worker is active in every level (skipping) and N < 128: rows leave one by one instead of as a box
+    N, P, iters, s = 96, 128 * 9, 16, 3
+    ptr, idx = inputs.graph_to_csr(inputs.complete(N))
+    ticks = np.ones((N, iters), np.uint64)
+    ticks[5, :] = 9
+    w = inputs.Workload(0, "dense-skip", N, P, iters, s=s, b=6, max_skip=3, max_ig=4, lr=0.05, momentum=0.0,
+                        weight_mode=inputs.STALE_LINEAR, grad_mode=inputs.GRAD_SYNTHETIC, in_ptr=ptr, in_idx=idx,
+                        ticks=ticks, grad_seed=4242)
+    w._p0 = np.random.default_rng(3).standard_normal(P).astype(np.float32)
+    g = GpuRun(w, hop.MIX_TENSOR)
+    tr = g.trace.to_arrays()
+    assert (tr["op"] == op.JUMP).sum() > 0 and (tr["op"] == op.IDLE).sum() > 0
+    assert all(g.h.level_stats(k)["kernel"] == hop.MIX_TENSOR for k in range(iters))
+    g.h.close()
+    check(w, iters, TOL_RUN, hop.MIX_TENSOR, perturb=True)
+    check(w, 1, TOL_STEP, hop.MIX_TENSOR, perturb=True)
+
+
 def test_cfg5_full_size_sampled_columns_first_levels():
     w = inputs.make_workload(5)
     cols = np.unique(np.concatenate([np.arange(0, w.P, 40009), [w.P - 1, w.P - 3, 127, 128, 255, 256]]))
