@@ -11,13 +11,13 @@
 // float32 in the epilogue where the row scaling 1/den_i is applied.
 //
 // Roles inside one persistent thread block (one per SM), tile = 128 parameter columns x all workers:
-//   warp 0      producer: the 16 raw X row pieces of a K-chunk, four TMA tile::gather4 loads (4 arbitrary rows of
-//               the ring per instruction; issuing one copy per row would be issue-bound: ~27 ns per copy and lane)
+//   warps 0, 2  producers: the 16 raw X row pieces of a K-chunk as four TMA tile::gather4 loads (4 arbitrary rows
+//               of the ring per instruction), two per warp: a warp issues at ~27 ns per row fetched (measured)
 //   warp 1      MMA issue (one elected lane): tcgen05.mma kind::tf32, M=128 (columns) x N=128 (workers) x K=8,
 //               A operand (X_hi / X_lo) from tensor memory, B operand (A^T, resident) from shared memory
 //   warp 3      gradient producer: one 2-D TMA box load of the tile's N x 128 piece of G into shared memory
 //   warps 4-7   converters: lane = column; read the raw chunk from shared memory, split hi/lo with
-//               cvt.rna.tf32, tcgen05.st into the A stages in tensor memory
+//               round-to-nearest TF32 splitting, tcgen05.st into the A stages in tensor memory
 //   warps 8-11  epilogue: tcgen05.ld both accumulators, add, release them, then y = acc/den - lr*g written over g
 //               in shared memory; the finished N x 128 tile goes to the output slot as one TMA box store (or
 //               one bulk row copy per active worker when some workers are idle in the level)
@@ -38,7 +38,7 @@ namespace {
 
 constexpr int kTile = 128;          // parameter columns per tile = MMA M
 constexpr int kChunk = 16;          // K rows per pipeline stage
-constexpr int kStages = 8;          // tensor-memory A stages; raw shared-memory stages: 3..8, chosen by the host
+constexpr int kStages = 8;          // tensor-memory A stages (power of two); raw shared-memory stages: 3..8, chosen by the host
 constexpr int kThreads = 12 * 32;
 constexpr uint32_t kSpin = 1u << 20;
 constexpr int kRawStageBytes = kChunk * kTile * 4;          // 8 KB
@@ -75,7 +75,11 @@ __device__ __forceinline__ void tma_tile2d(void* dst, const CUtensorMap* map, in
     asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  ::"r"(s32(dst)), "l"(map), "r"(x), "r"(y), "r"(s32(bar)) : "memory");
 }
-__device__ __forceinline__ uint32_t to_tf32(float x) { uint32_t r; asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x)); return r; }
+// Round to TF32 (10 explicit mantissa bits), nearest with ties away from zero, on the integer pipe: add half
+// an ulp to the magnitude and clear the 13 low bits.  Same result as cvt.rna.tf32.f32 for finite inputs, but
+// that conversion instruction issues at a fraction of the integer rate and made the converter warps the
+// slowest stage (measured).
+__device__ __forceinline__ uint32_t to_tf32(float x) { return (__float_as_uint(x) + 0x1000u) & 0xFFFFE000u; }
 
 // Shared-memory matrix descriptor, K-major, no swizzle: 8x(16 B) core matrices; leading-dimension byte
 // offset = distance between core matrices adjacent in K, stride byte offset = distance between 8-row
@@ -102,6 +106,14 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16
                  ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]),
                  "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+                 "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+                 ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]),
+                 "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]),
+                 "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]),
+                 "r"(v[30]), "r"(v[31]) : "memory");
+}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     uint32_t r[32];
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
@@ -121,6 +133,8 @@ struct TcSmem {                       // control block at the start of dynamic s
     uint32_t tmem_base;
     int abort_flag;
     int epi_fail;
+    uint32_t active_mask[4], g_mask[4];   // bit i of word i/32: worker i writes a result / applies a gradient
+    alignas(16) float inv_den[128];
     HopTcRow rows[128];
 };
 
@@ -141,7 +155,7 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
     volatile int* abort_flag = &cb->abort_flag;
 
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) { mb_init(&cb->raw_full[s], 1); mb_init(&cb->raw_empty[s], 4); mb_init(&cb->a_full[s], 4); mb_init(&cb->a_empty[s], 1); }
+        for (int s = 0; s < kStages; ++s) { mb_init(&cb->raw_full[s], 2); mb_init(&cb->raw_empty[s], 4); mb_init(&cb->a_full[s], 4); mb_init(&cb->a_empty[s], 1); }
         mb_init(&cb->acc_full, 1); mb_init(&cb->acc_empty, 4); mb_init(&cb->w_full, 1);
         mb_init(&cb->g_full, 1); mb_init(&cb->g_empty, 1);
         cb->abort_flag = 0;
@@ -149,7 +163,12 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    for (int i = tid; i < 128; i += kThreads) cb->rows[i] = tbl[i];
+    for (int i = tid; i < 128; i += kThreads) { cb->rows[i] = tbl[i]; cb->inv_den[i] = tbl[i].inv_den; }
+    if (tid < 4) {
+        uint32_t am = 0, gm = 0;
+        for (int i = 0; i < 32; ++i) { am |= (uint32_t)(tbl[tid * 32 + i].out_row >= 0) << i; gm |= (uint32_t)(tbl[tid * 32 + i].g_row >= 0) << i; }
+        cb->active_mask[tid] = am; cb->g_mask[tid] = gm;
+    }
     if (warp == 2) {   // tensor-memory allocation: all 512 columns, by one warp, which also frees them
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(s32(&cb->tmem_base)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -160,26 +179,29 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
     const uint32_t tmem = cb->tmem_base;
     const uint32_t kDhi = 0, kDlo = 128, kA0 = 256;
 
-    if (warp == 0) {
-        // ------------------------------------------------ producer
-        if (lane == 0) {
+    if (warp == 0 || warp == 2) {
+        // ------------------------------------------------ producers: two warps, two gather4 loads each per chunk
+        // (a warp issues its TMA loads one after the other, ~27 ns per row fetched: one warp alone cannot keep up)
+        const int half = warp >> 1;
+        if (warp == 0 && lane == 0) {
             mb_expect_tx(&cb->w_full, (uint32_t)Kpad * 512u);
             bulk_g2s(Wsm, Wk, (uint32_t)Kpad * 512u, &cb->w_full);
         }
-        int64_t q = 0;
+        int s = 0;             // raw stage and its phase bit, advanced by hand (raw_stages is not a power of two)
+        uint32_t ph = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
-            for (int c = 0; c < nchunks && ok; ++c, ++q) {
-                const int s = (int)(q % raw_stages);
-                const uint32_t ph = (uint32_t)((q / raw_stages) & 1);
+            for (int c = 0; c < nchunks && ok; ++c) {
                 if (!mb_wait(&cb->raw_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
-                if (lane == 0) mb_expect_tx(&cb->raw_full[s], kRawStageBytes);
+                if (lane == 0) mb_expect_tx(&cb->raw_full[s], kRawStageBytes / 2);
                 __syncwarp();
-                if (lane < kChunk / 4) {
-                    const int u = c * kChunk + lane * 4;
-                    tma_gather4(raw + (size_t)s * (kChunk * kTile) + lane * 4 * kTile, &mapX, (int)(tile * kTile),
+                if (lane < 2) {
+                    const int r4 = half * 2 + lane;                 // which group of four rows of the chunk
+                    const int u = c * kChunk + r4 * 4;
+                    tma_gather4(raw + (size_t)s * (kChunk * kTile) + r4 * 4 * kTile, &mapX, (int)(tile * kTile),
                                 src_row[u], src_row[u + 1], src_row[u + 2], src_row[u + 3], &cb->raw_full[s]);
                 }
+                if (++s == raw_stages) { s = 0; ph ^= 1u; }
             }
         }
         if (!ok && lane == 0) { atomicCAS(err_word, 0, ERR_TC_WAIT | 1); cb->abort_flag = 1; }
@@ -234,36 +256,53 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         int64_t q = 0;
         bool ok = true;
+        // The tensor-memory store of chunk q is left in flight while chunk q+1 is fetched from shared memory;
+        // chunk q is published to the MMA warp (a_full) once tcgen05.wait::st has covered it.
+        int pending = -1;
+        auto publish = [&]() {
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            fence_before();
+            __syncwarp();
+            if (lane == 0) mb_arrive(&cb->a_full[pending]);
+            pending = -1;
+        };
+        int rs = 0;
+        uint32_t rph = 0;
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
             for (int c = 0; c < nchunks; ++c, ++q) {
-                const int s = (int)(q % kStages), rs = (int)(q % raw_stages);
-                if (!mb_wait(&cb->raw_full[rs], (uint32_t)((q / raw_stages) & 1), abort_flag) ||
-                    !mb_wait(&cb->a_empty[s], (uint32_t)(((q / kStages) & 1) ^ 1), abort_flag)) { ok = false; break; }
-                fence_after();
+                const int s = (int)(q & (kStages - 1));
+                if (pending >= 0 && !mb_try(&cb->raw_full[rs], rph)) publish();   // nothing to overlap with
+                if (!mb_wait(&cb->raw_full[rs], rph, abort_flag)) { ok = false; break; }
                 const float* r = raw + (size_t)rs * (kChunk * kTile) + col;
-                uint32_t hi[kChunk], lo[kChunk];
+                float x[kChunk];
+#pragma unroll
+                for (int u = 0; u < kChunk; ++u) x[u] = r[u * kTile];
+                if (pending >= 0) publish();
+                if (!mb_wait(&cb->a_empty[s], (uint32_t)(((q / kStages) & 1) ^ 1), abort_flag)) { ok = false; break; }
+                fence_after();
+                uint32_t v[2 * kChunk];                      // hi in columns 0..15 of the stage, lo in 16..31
 #pragma unroll
                 for (int u = 0; u < kChunk; ++u) {
-                    const float x = r[u * kTile];
-                    hi[u] = to_tf32(x);
-                    lo[u] = to_tf32(x - __uint_as_float(hi[u]));
+                    v[u] = to_tf32(x[u]);
+                    v[kChunk + u] = to_tf32(x[u] - __uint_as_float(v[u]));
                 }
-                const uint32_t a_hi = tmem + lane_base + kA0 + s * 32;
-                tmem_st16(a_hi, hi);
-                tmem_st16(a_hi + 16, lo);
-                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                fence_before();
                 __syncwarp();
-                if (lane == 0) { mb_arrive(&cb->a_full[s]); mb_arrive(&cb->raw_empty[rs]); }
+                if (lane == 0) mb_arrive(&cb->raw_empty[rs]);   // the raw chunk is in registers
+                tmem_st32(tmem + lane_base + kA0 + s * 32, v);
+                pending = s;
+                if (++rs == raw_stages) { rs = 0; rph ^= 1u; }
             }
         }
+        if (pending >= 0) publish();
         if (!ok && lane == 0) { atomicCAS(err_word, 0, ERR_TC_WAIT | 3); cb->abort_flag = 1; }
     } else if (warp >= 8) {
         // ------------------------------------------------ epilogue (lane quarter = warp % 4)
         const int col = (warp - 8) * 32 + lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        bool has_g = false;
-        for (int i = 0; i < 128; ++i) has_g |= (cb->rows[i].g_row >= 0);
+        uint32_t am[4], gm[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { am[k] = cb->active_mask[k]; gm[k] = cb->g_mask[k]; }
+        const bool has_g = (gm[0] | gm[1] | gm[2] | gm[3]) != 0;
         int64_t tcount = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++tcount) {
@@ -289,12 +328,22 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                     // y = acc/den - lr*g replaces g in the shared tile (column-per-thread: conflict-free), then the
                     // tile leaves through the copy engine: per-thread 4-byte global stores of 128 different rows
                     // were the slowest part of the kernel by far (measured)
+                    // Batches of 8 rows with every shared-memory load ahead of the batch's stores: the compiler
+                    // cannot prove that the stores do not alias the tables, and a load-store-load chain per row
+                    // cost ~100 cycles per row (measured).
 #pragma unroll
-                    for (int i = 0; i < 128; ++i) {
-                        const HopTcRow rw = cb->rows[i];
-                        if (rw.out_row >= 0) {
-                            const float g = (rw.g_row >= 0) ? Gsm[i * kTile + col] : 0.f;
-                            Gsm[i * kTile + col] = fmaf(-lr, g, acc[i] * rw.inv_den);
+                    for (int b = 0; b < 128; b += 8) {
+                        const float4 s0 = *reinterpret_cast<const float4*>(&cb->inv_den[b]);
+                        const float4 s1 = *reinterpret_cast<const float4*>(&cb->inv_den[b + 4]);
+                        const float sc[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+                        float g[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) g[i] = Gsm[(b + i) * kTile + col];   // stale but unused when the row has no gradient
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int r = b + i;
+                            const float gv = ((gm[r >> 5] >> (r & 31)) & 1u) ? g[i] : 0.f;
+                            if ((am[r >> 5] >> (r & 31)) & 1u) Gsm[r * kTile + col] = fmaf(-lr, gv, acc[r] * sc[i]);
                         }
                     }
                 }
