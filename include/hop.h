@@ -177,9 +177,10 @@ int hop_step_host(hop_ctx* ctx, const int32_t* op, const int64_t* ptr, const int
  * a code in the top byte and a detail in the rest). */
 int hop_read_status(hop_ctx* ctx, int32_t* device_error_word);
 
-/* out[8] (host) for a level of the loaded trace: distinct consumed slices U_k, NORMAL records,
- * JUMP records, consumed entries sum_i |C_{i,k}|, tile width chosen, kernel chosen, staged rows,
- * algorithmic bytes of the mix-update kernel. */
+/* out[10] (host) for a level of the loaded trace: distinct consumed slices U_k, NORMAL records,
+ * JUMP records, consumed entries sum_i |C_{i,k}|, tile width chosen, kernel chosen (hop_mix_kernel),
+ * staged rows, algorithmic bytes of the mix-update kernel, tensor-core flops issued by the dense
+ * path (0 for the other kernels), K padded to the MMA chunk (dense path). */
 int hop_level_stats(hop_ctx* ctx, int32_t level, int64_t* out);
 /* Per-kernel-class timing (tracing aid).  While enabled, hop_step / hop_step_host bracket each
  * kernel class with CUDA events on the bound stream.  hop_timing_read synchronises the stream and

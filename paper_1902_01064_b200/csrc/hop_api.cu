@@ -38,6 +38,7 @@ struct hop_ctx {
     int32_t* d_tcsrc = nullptr;
     alignas(64) unsigned char tc_mapX[128], tc_mapG[128], tc_mapY[8 * 128];   // TMA tensor maps over X, G, output slots
     int32_t tc_slots = 0;
+    bool tc_maps_ready = false;
     int32_t* d_i32 = nullptr;       // src_row and grad_workers of all levels
     HopRecord* d_rec = nullptr;
     HopEntry* d_ent = nullptr;
@@ -201,6 +202,7 @@ extern "C" int hop_bind_buffers(hop_ctx* c, float* X, float* M, float* G, void* 
     const int rc = ensure_device(c);
     if (rc) return rc;
     c->X = X; c->M = M; c->G = G; c->stream = (cudaStream_t)stream; c->bound = true;
+    c->tc_maps_ready = false;
     return HOP_OK;
 }
 
@@ -288,6 +290,8 @@ static int plan_level(hop_ctx* c, HopLevelHost& L, bool allow_tensor = true) {
     return HOP_OK;
 }
 
+static int ensure_tc_maps(hop_ctx* c);
+
 extern "C" int hop_load_trace(hop_ctx* c, const hop_trace* t) {
     if (!c || !t) return HOP_E_ARG;
     if (!c->bound) HOP_FAIL(c, HOP_E_STATE, "hop_load_trace: bind buffers first");
@@ -335,10 +339,8 @@ extern "C" int hop_load_trace(hop_ctx* c, const hop_trace* t) {
         HOP_CUDA(c, cudaMemcpyAsync(c->d_tcw, h_tcw.data(), h_tcw.size() * sizeof(float), cudaMemcpyHostToDevice, c->stream));
         HOP_CUDA(c, cudaMemcpyAsync(c->d_tcrows, h_tcrows.data(), h_tcrows.size() * sizeof(HopTcRow), cudaMemcpyHostToDevice, c->stream));
         HOP_CUDA(c, cudaMemcpyAsync(c->d_tcsrc, h_tcsrc.data(), h_tcsrc.size() * sizeof(int32_t), cudaMemcpyHostToDevice, c->stream));
-        c->tc_slots = (c->s + 1 <= 8) ? c->s + 1 : 0;
-        const int me = hop_dense_tc_make_maps(c->X, (int64_t)c->g.N * (c->s + 1), c->G, c->g.N, c->P, c->tc_mapX, c->tc_mapG,
-                                              c->tc_mapY, c->tc_slots);
-        if (me) HOP_FAIL(c, HOP_E_CUDA, std::string("tensor map for the dense path: ") + cudaGetErrorString((cudaError_t)me));
+        const int mrc = ensure_tc_maps(c);
+        if (mrc) return mrc;
     }
     HOP_CUDA(c, cudaStreamSynchronize(c->stream));   // the host vectors go out of scope
     c->levels = std::move(levels);
@@ -374,7 +376,19 @@ static int mark(hop_ctx* c, size_t* idx) {
     c->spans.push_back({t0, t1, (kind), (int64_t)(bytes)}); } } while (0)
 
 // Enqueues the kernels of one level.
-static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv) {
+struct TcPtrs { const float* w; const HopTcRow* rows; const int32_t* src; };   // device tables of the dense path
+
+static int ensure_tc_maps(hop_ctx* c) {
+    if (c->tc_maps_ready) return HOP_OK;
+    c->tc_slots = (c->s + 1 <= 8) ? c->s + 1 : 0;
+    const int me = hop_dense_tc_make_maps(c->X, (int64_t)c->g.N * (c->s + 1), c->G, c->g.N, c->P, c->tc_mapX, c->tc_mapG,
+                                          c->tc_mapY, c->tc_slots);
+    if (me) HOP_FAIL(c, HOP_E_CUDA, std::string("tensor map for the dense path: ") + cudaGetErrorString((cudaError_t)me));
+    c->tc_maps_ready = true;
+    return HOP_OK;
+}
+
+static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, const TcPtrs& tc) {
     size_t t0 = 0, t1 = 0;
     HopLaunchCfg cfg{};
     cfg.X = c->X; cfg.M = c->M; cfg.G = c->G; cfg.P = c->P; cfg.N = c->g.N; cfg.s = c->s;
@@ -402,7 +416,7 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv) {
         if (L.kernel == HOP_MIX_TENSOR)
             e = hop_launch_mix_dense_tc(cfg, c->tc_mapX, c->tc_mapG,
                                         (L.nA == c->g.N && c->tc_slots > 0) ? c->tc_mapY + 128 * ((lv.level + 1) % (c->s + 1)) : nullptr,
-                                        c->d_tcw + L.off_tcw, c->d_tcrows + L.off_tcrows, c->d_tcsrc + L.off_tcsrc, L.Kpad);
+                                        tc.w, tc.rows, tc.src, L.Kpad);
         else
             e = (L.kernel == HOP_MIX_BULK) ? hop_launch_mix_bulk(cfg, lv) : hop_launch_mix_staged(cfg, lv);
         c->launches += 1;
@@ -428,7 +442,7 @@ extern "C" int hop_step(hop_ctx* c) {
     const HopLevelHost& L = c->levels[c->level];
     HopLevelDev lv{c->d_i32 + L.off_src, c->d_rec + L.off_rec, c->d_ent + L.off_ent, c->d_i32 + L.off_gw,
                    L.U, L.nA, L.nG, c->level};
-    rc = run_level(c, L, lv);
+    rc = run_level(c, L, lv, TcPtrs{c->d_tcw + L.off_tcw, c->d_tcrows + L.off_tcrows, c->d_tcsrc + L.off_tcsrc});
     if (rc) return rc;
     for (const HopRecord& r : L.recs) c->newest[r.worker] = c->level + 1;
     c->level += 1;
@@ -454,12 +468,19 @@ extern "C" int hop_step_host(hop_ctx* c, const int32_t* op, const int64_t* ptr, 
     if (rc) return rc;
     HopLevelHost L;
     hop_build_level(c->g, c->s, k, op, ptr, nbr, ver, num, den, L);
-    rc = plan_level(c, L, false);   // the streaming path uploads only the general kernels' tables
+    rc = plan_level(c, L);
     if (rc) return rc;
+    const bool tcl = L.kernel == HOP_MIX_TENSOR;
+    if (tcl && (rc = ensure_tc_maps(c))) return rc;
     // pack [src_row | grad_workers | recs | ents] into one pinned buffer, one H2D copy
     const size_t b_src = L.src_row.size() * 4, b_gw = L.grad_workers.size() * 4;
     const size_t o_gw = b_src, o_rec = (o_gw + b_gw + 15) / 16 * 16, b_rec = L.recs.size() * sizeof(HopRecord);
-    const size_t o_ent = o_rec + b_rec, b_ent = L.ents.size() * sizeof(HopEntry), total = std::max<size_t>(16, o_ent + b_ent);
+    const size_t o_ent = o_rec + b_rec, b_ent = L.ents.size() * sizeof(HopEntry);
+    // dense path: weight numerators (16-byte aligned for the bulk copy), row table, padded slice rows
+    const size_t o_tcw = (o_ent + b_ent + 127) / 128 * 128, b_tcw = tcl ? L.tc_w.size() * sizeof(float) : 0;
+    const size_t o_tcr = o_tcw + b_tcw, b_tcr = tcl ? L.tc_rows.size() * sizeof(HopTcRow) : 0;
+    const size_t o_tcs = (o_tcr + b_tcr + 15) / 16 * 16, b_tcs = tcl ? L.tc_src.size() * sizeof(int32_t) : 0;
+    const size_t total = std::max<size_t>(16, o_tcs + b_tcs);
     if (total > c->stage_cap) {
         if (c->d_stage) cudaFree(c->d_stage);
         if (c->h_stage) cudaFreeHost(c->h_stage);
@@ -480,11 +501,14 @@ extern "C" int hop_step_host(hop_ctx* c, const int32_t* op, const int64_t* ptr, 
     if (b_gw) std::memcpy(h + o_gw, L.grad_workers.data(), b_gw);
     if (b_rec) std::memcpy(h + o_rec, L.recs.data(), b_rec);
     if (b_ent) std::memcpy(h + o_ent, L.ents.data(), b_ent);
+    if (b_tcw) std::memcpy(h + o_tcw, L.tc_w.data(), b_tcw);
+    if (b_tcr) std::memcpy(h + o_tcr, L.tc_rows.data(), b_tcr);
+    if (b_tcs) std::memcpy(h + o_tcs, L.tc_src.data(), b_tcs);
     HOP_CUDA(c, cudaMemcpyAsync(c->d_stage, h, total, cudaMemcpyHostToDevice, c->stream));
     unsigned char* d = (unsigned char*)c->d_stage;
     HopLevelDev lv{(const int32_t*)d, (const HopRecord*)(d + o_rec), (const HopEntry*)(d + o_ent), (const int32_t*)(d + o_gw),
                    L.U, L.nA, L.nG, k};
-    rc = run_level(c, L, lv);
+    rc = run_level(c, L, lv, TcPtrs{(const float*)(d + o_tcw), (const HopTcRow*)(d + o_tcr), (const int32_t*)(d + o_tcs)});
     if (rc) return rc;
     c->newest = newest;
     c->level += 1;
@@ -557,6 +581,8 @@ extern "C" int hop_level_stats(hop_ctx* c, int32_t level, int64_t* out) {
     const HopLevelHost& L = c->levels[level];
     out[0] = L.U; out[1] = L.nG; out[2] = L.nJump; out[3] = L.sumC; out[4] = L.tile_w; out[5] = L.kernel;
     out[6] = L.stage_rows; out[7] = L.alg_bytes;
+    out[8] = L.kernel == HOP_MIX_TENSOR ? (int64_t)2 * 2 * 128 * L.Kpad * c->P : 0;   // two TF32 passes, M x N x K = P x 128 x Kpad
+    out[9] = L.Kpad;
     return HOP_OK;
 }
 

@@ -191,9 +191,10 @@ class Hop:
         return w.value
 
     def level_stats(self, level):
-        out = np.zeros(8, np.int64)
+        out = np.zeros(10, np.int64)
         self._chk(lib.hop_level_stats(self.h, level, _ptr(out)))
-        return dict(zip(("U", "normal", "jump", "entries", "tile_w", "kernel", "stage_rows", "alg_bytes"), out.tolist()))
+        return dict(zip(("U", "normal", "jump", "entries", "tile_w", "kernel", "stage_rows", "alg_bytes", "mma_flops", "k_padded"),
+                        out.tolist()))
 
     def timing_enable(self, on=True):
         self._chk(lib.hop_timing_enable(self.h, 1 if on else 0))

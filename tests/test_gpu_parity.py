@@ -254,8 +254,10 @@ def test_in_place_ring_hazard_single_slot_and_stale_reads():
             check(w, iters, TOL_RUN, kernel, perturb=True)
 
 
-def test_streaming_levels_equal_preloaded_trace_bitwise():
-    w = inputs.make_workload(3, P=2048, iters=40)
+@pytest.mark.parametrize("cfg,P,iters", [(3, 2048, 40), (5, 1536, 8)])
+def test_streaming_levels_equal_preloaded_trace_bitwise(cfg, P, iters):
+    # configuration 5 goes through the tensor-core kernel in both modes
+    w = inputs.make_workload(cfg, P=P, iters=iters)
     a = GpuRun(w)
     ref = a.run(w.iters)
     b = GpuRun(w)
