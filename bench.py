@@ -29,9 +29,11 @@ if ROOT not in sys.path:
 METRIC = "worker_iterations_per_s"
 UNIT = "worker-iterations/s"
 PROBE = 1024
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the mix-update kernel from the ncu capture
-# summarised under profiles/ (a smaller P scaled by columns), or None when the kernel changed since.
-NCU_TRAFFIC = {}
+# dram__bytes_read.sum + dram__bytes_write.sum (bytes, per launch, averaged over the trace) of the mix-update kernel
+# from the ncu captures summarised under profiles/: taken at a smaller parameter count and scaled by the number of
+# columns (traffic is proportional to columns at a fixed trace).  Dropped to None whenever the kernel changes.
+NCU_TRAFFIC = {(4, 25_600_000): 23.52e9,      # profiles/mix_bulk_kernel_cfg4.md, section 2b (all 50 levels)
+               (5, 8_000_000): 0.98 * 12.96e9}  # profiles/mix_dense_tc_kernel_cfg5.md, section 2 (ratio of two levels)
 
 
 def shard_columns(P: int, n: int, r: int, unit: int = 128):
@@ -322,7 +324,7 @@ def main():
     ach = tim["mix_bytes"] / (tim["ms_mix"] * 1e-3) / 1e9 if tim["ms_mix"] > 0 else 0.0
     traffic = NCU_TRAFFIC.get((args.config, P_global))
     roofline = {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
-                "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": "+".join(kname[k] for k in kernels),
+                "traffic": traffic, "traffic_unit": "bytes per launch", "peak_kind": f"of {peak_kind}", "kernel": "+".join(kname[k] for k in kernels),
                 "launches": mix_launches, "avg_launch_ms": tim["ms_mix"] / max(1, mix_launches),
                 "alg_bytes_per_launch": tim["mix_bytes"] / max(1, mix_launches),
                 "frac_of_nominal_8TBs": ach / 8000.0,
