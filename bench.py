@@ -286,7 +286,7 @@ def main():
             per_level.append((np.ascontiguousarray(tr["op"][k]), (tr["ptr"][k * N:(k + 1) * N + 1] - a).astype(np.int64),
                               np.ascontiguousarray(tr["nbr"][a:b]), np.ascontiguousarray(tr["ver"][a:b]),
                               np.ascontiguousarray(tr["num"][a:b]), np.ascontiguousarray(tr["den"][k])))
-        probe = np.zeros(PROBE, np.float32)
+        probe = np.zeros(min(PROBE, w.P), np.float32)
         n_e2e = min(args.steps, w.iters)
         for k in range(min(3, w.iters)):
             h.step_host(*per_level[k], probe)

@@ -248,24 +248,30 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
     constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
-        const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
-        const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+        const uint64_t p0 = (uint64_t)M0 * c0, p1 = (uint64_t)M1 * c2;     // one wide multiply each
+        const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+        const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
         c0 = hi1 ^ c1 ^ k0; c1 = lo1; c2 = hi0 ^ c3 ^ k1; c3 = lo0;
         k0 += W0; k1 += W1;
     }
     o[0] = c0; o[1] = c1; o[2] = c2; o[3] = c3;
 }
-// Box-Muller on 23-bit uniforms u = (n + 1/2) / 2^23 (exact in float32).  The hardware approximations
-// __logf / __sincosf are used on purpose: their error (<= 3 ulp for the logarithm, <= 2^-21.4 absolute
-// for sine and cosine on [-pi, pi]) changes a normal deviate by < 3e-6, i.e. a parameter by < 1e-9
-// per step after scaling by sigma and the learning rate, and the kernel is arithmetic-bound otherwise.
-__device__ __forceinline__ void box_muller(uint32_t ra, uint32_t rb, float& z0, float& z1) {
-    const float u1 = (float)(((ra >> 9) << 1) | 1u) * 5.9604644775390625e-08f;      // (2n+1) * 2^-24
-    const float two_u2 = (float)(((rb >> 9) << 1) | 1u) * 1.1920928955078125e-07f;  // 2 * u2 in (0, 2)
-    const float rad = sqrtf(-2.0f * __logf(u1));
-    float sn, cs;
-    __sincosf((two_u2 - 1.0f) * 3.14159265358979323846f, &sn, &cs);                  // angle - pi in (-pi, pi)
-    z0 = -rad * cs; z1 = -rad * sn;                                                  // cos(a) = -cos(a - pi)
+// Box-Muller on 23-bit uniforms u = (n + 1/2) / 2^23 (exact in float32), scaled by sigma.  The kernel is
+// instruction-bound, so: the uniforms are built by placing the 23 random bits in the mantissa of a float in
+// [1, 2) (no integer-to-float conversion); the hardware approximations lg2 / sqrt / sin / cos are used on purpose
+// (error <= 3 ulp for the logarithm, 2 ulp for the root, <= 2^-21.4 absolute for sine and cosine on [-pi, pi]:
+// a normal deviate moves by < 3e-6, a parameter by < 1e-9 per step after scaling by sigma and the learning rate).
+__device__ __forceinline__ void box_muller(uint32_t ra, uint32_t rb, float sigma, float& z0, float& z1) {
+    const float f1 = __uint_as_float(0x3f800000u | (ra >> 9));        // 1 + n1 * 2^-23
+    const float f2 = __uint_as_float(0x3f800000u | (rb >> 9));        // 1 + n2 * 2^-23
+    const float u1 = (f1 - 1.0f) + 5.9604644775390625e-08f;           // (n1 + 1/2) * 2^-23, exact
+    const float t = fmaf(2.0f, f2 - 1.5f, 1.1920928955078125e-07f);   // 2*u2 - 1 in (-1, 1), exact
+    float l2, rad, sn, cs;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(l2) : "f"(u1));
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rad) : "f"(l2 * -1.3862943611198906f));   // sqrt(-2 ln u1)
+    __sincosf(t * 3.14159265358979323846f, &sn, &cs);                 // angle - pi in (-pi, pi)
+    rad *= -sigma;                                                    // cos(a) = -cos(a - pi), sin likewise
+    z0 = rad * cs; z1 = rad * sn;
 }
 
 __global__ void __launch_bounds__(256)
@@ -278,13 +284,13 @@ synth_grad_kernel(float* __restrict__ G, int64_t P, HopLevelDev lv, uint32_t k0,
     const uint64_t gq = (uint64_t)(col_offset / 4 + q);
     philox4x32_10((uint32_t)gq, (uint32_t)worker, (uint32_t)lv.level, 6u, k0, k1, o);
     float z[4];
-    box_muller(o[0], o[1], z[0], z[1]);
-    box_muller(o[2], o[3], z[2], z[3]);
+    box_muller(o[0], o[1], sigma, z[0], z[1]);
+    box_muller(o[2], o[3], sigma, z[2], z[3]);
     float* dst = G + (int64_t)worker * P + c;
     if (c + 4 <= P && (P & 3) == 0) {
-        *reinterpret_cast<float4*>(dst) = make_float4(sigma * z[0], sigma * z[1], sigma * z[2], sigma * z[3]);
+        *reinterpret_cast<float4*>(dst) = make_float4(z[0], z[1], z[2], z[3]);
     } else {
-        for (int e = 0; e < 4 && c + e < P; ++e) dst[e] = sigma * z[e];
+        for (int e = 0; e < 4 && c + e < P; ++e) dst[e] = z[e];
     }
 }
 

@@ -10,6 +10,9 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
+    # the binding refuses to import without the shared library: build it in-tree when it is missing or stale
+    from paper_1902_01064_b200 import build
+    build.build()
 
 
 def pytest_collection_modifyitems(config, items):
