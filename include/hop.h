@@ -95,6 +95,7 @@ typedef enum hop_option {
     HOP_OPT_MIX_KERNEL = 8,   /* hop_mix_kernel (default AUTO)                                      */
     HOP_OPT_COL_OFFSET = 9,   /* global index of local parameter 0 when P is a shard of a larger    */
                               /* vector (multiple of 4); only the synthetic gradient reads it       */
+    HOP_OPT_USE_GRAPH = 10,   /* hop_run may replay a captured CUDA graph (default 1)                    */
     HOP_OPT_BACKUP_OF_WORKER = 1000 /* key = 1000 + i sets N_buw(i) of one worker (Fig. alg4)       */
 } hop_option;
 
@@ -165,6 +166,12 @@ int hop_set_level(hop_ctx* ctx, int32_t level);
  * then the fused gather-mix-update writing slot k+1, then (CSR SVM) the sparse apply.
  * Asynchronous; HOP_E_STATE past the end of the trace. */
 int hop_step(hop_ctx* ctx);
+/* Executes the next n_levels levels of the loaded trace.  When the bound stream is not the default
+ * stream, the levels are captured once into a CUDA graph (cached per (first level, n_levels); dropped
+ * by any bind / option / trace change) and replayed, which removes most of the per-kernel launch cost
+ * that dominates small problems.  Falls back to a plain loop of hop_step on the default stream, while
+ * timing is enabled, with HOP_GRAD_EXTERNAL, or with HOP_OPT_USE_GRAPH = 0.  Asynchronous. */
+int hop_run(hop_ctx* ctx, int32_t n_levels);
 /* Same for one level handed in from the host (streaming use: the protocol decides level by
  * level): validates the records, uploads them from a pinned staging buffer, executes the level,
  * copies the first probe_len floats of worker 0's new version into probe_dst (host, may be NULL)

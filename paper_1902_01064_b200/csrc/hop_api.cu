@@ -5,6 +5,8 @@
 #include <cmath>
 #include <cstring>
 #include <string>
+#include <map>
+#include <utility>
 #include <vector>
 
 #include "hop_internal.h"
@@ -39,6 +41,9 @@ struct hop_ctx {
     alignas(64) unsigned char tc_mapX[128], tc_mapG[128], tc_mapY[8 * 128];   // TMA tensor maps over X, G, output slots
     int32_t tc_slots = 0;
     bool tc_maps_ready = false;
+    // hop_run: instantiated CUDA graphs of level ranges, keyed by (first level, count)
+    bool use_graph = true;
+    std::map<std::pair<int32_t, int32_t>, cudaGraphExec_t> graphs;
     int32_t* d_i32 = nullptr;       // src_row and grad_workers of all levels
     HopRecord* d_rec = nullptr;
     HopEntry* d_ent = nullptr;
@@ -112,7 +117,14 @@ extern "C" int hop_create(hop_ctx** out, const int32_t* in_ptr, const int32_t* i
     return HOP_OK;
 }
 
+// Kernel arguments (pointers, learning rate, tables) are baked into captured graphs: drop them on any change.
+static void drop_graphs(hop_ctx* c) {
+    for (auto& kv : c->graphs) cudaGraphExecDestroy(kv.second);
+    c->graphs.clear();
+}
+
 static void free_trace_tables(hop_ctx* c) {
+    drop_graphs(c);
     if (c->d_i32) cudaFree(c->d_i32);
     if (c->d_rec) cudaFree(c->d_rec);
     if (c->d_ent) cudaFree(c->d_ent);
@@ -140,6 +152,8 @@ extern "C" int hop_destroy(hop_ctx* c) {
 
 extern "C" int hop_set_option(hop_ctx* c, int key, double v) {
     if (!c) return HOP_E_ARG;
+    drop_graphs(c);
+    if (key == HOP_OPT_USE_GRAPH) { c->use_graph = v != 0.0; return HOP_OK; }
     if (key >= HOP_OPT_BACKUP_OF_WORKER) {
         const int i = key - HOP_OPT_BACKUP_OF_WORKER;
         if (i >= c->g.N) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: worker index out of range");
@@ -203,6 +217,7 @@ extern "C" int hop_bind_buffers(hop_ctx* c, float* X, float* M, float* G, void* 
     if (rc) return rc;
     c->X = X; c->M = M; c->G = G; c->stream = (cudaStream_t)stream; c->bound = true;
     c->tc_maps_ready = false;
+    drop_graphs(c);
     return HOP_OK;
 }
 
@@ -446,6 +461,56 @@ extern "C" int hop_step(hop_ctx* c) {
     if (rc) return rc;
     for (const HopRecord& r : L.recs) c->newest[r.worker] = c->level + 1;
     c->level += 1;
+    return HOP_OK;
+}
+
+static int enqueue_level(hop_ctx* c, int32_t k) {
+    const HopLevelHost& L = c->levels[k];
+    HopLevelDev lv{c->d_i32 + L.off_src, c->d_rec + L.off_rec, c->d_ent + L.off_ent, c->d_i32 + L.off_gw, L.U, L.nA, L.nG, k};
+    return run_level(c, L, lv, TcPtrs{c->d_tcw + L.off_tcw, c->d_tcrows + L.off_tcrows, c->d_tcsrc + L.off_tcsrc});
+}
+
+extern "C" int hop_run(hop_ctx* c, int32_t n_levels) {
+    if (!c) return HOP_E_ARG;
+    if (!c->bound || !c->loaded) HOP_FAIL(c, HOP_E_STATE, "hop_run: bind buffers and load a trace first");
+    if (n_levels < 0 || c->level + n_levels > (int32_t)c->levels.size()) HOP_FAIL(c, HOP_E_STATE, "hop_run: past the end of the trace");
+    if (n_levels == 0) return HOP_OK;
+    int rc = check_mode(c);
+    if (rc) return rc;
+    const int32_t first = c->level;
+    // Graph replay needs a capturable stream (not the legacy default stream), no per-kernel event timing,
+    // and a gradient source that is part of the library (an external G changes between levels).
+    const bool graph = c->use_graph && c->stream != nullptr && !c->timing && c->grad_mode != HOP_GRAD_EXTERNAL && n_levels > 1;
+    if (!graph) {
+        for (int32_t k = first; k < first + n_levels; ++k)
+            if ((rc = enqueue_level(c, k))) return rc;
+    } else {
+        auto key = std::make_pair(first, n_levels);
+        auto it = c->graphs.find(key);
+        if (it == c->graphs.end()) {
+            const int64_t launches_before = c->launches;
+            HOP_CUDA(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeRelaxed));
+            for (int32_t k = first; k < first + n_levels && !rc; ++k) rc = enqueue_level(c, k);
+            cudaGraph_t g = nullptr;
+            const cudaError_t ce = cudaStreamEndCapture(c->stream, &g);
+            c->launches = launches_before;
+            if (rc) { if (g) cudaGraphDestroy(g); return rc; }
+            if (ce != cudaSuccess) { c->err = std::string("hop_run: stream capture: ") + cudaGetErrorString(ce); return HOP_E_CUDA; }
+            cudaGraphExec_t ex = nullptr;
+            const cudaError_t ie = cudaGraphInstantiate(&ex, g, 0);
+            cudaGraphDestroy(g);
+            if (ie != cudaSuccess) { c->err = std::string("hop_run: graph instantiation: ") + cudaGetErrorString(ie); return HOP_E_CUDA; }
+            it = c->graphs.emplace(key, ex).first;
+        }
+        HOP_CUDA(c, cudaGraphLaunch(it->second, c->stream));
+        for (int32_t k = first; k < first + n_levels; ++k) {
+            const HopLevelHost& L = c->levels[k];
+            c->launches += (L.nA > 0) + (L.nG > 0 ? (c->grad_mode == HOP_GRAD_SVM_DENSE ? 2 : c->grad_mode == HOP_GRAD_SVM_CSR ? 2 : 1) : 0);
+        }
+    }
+    for (int32_t k = first; k < first + n_levels; ++k)
+        for (const HopRecord& r : c->levels[k].recs) c->newest[r.worker] = k + 1;
+    c->level = first + n_levels;
     return HOP_OK;
 }
 

@@ -453,7 +453,7 @@ int hop_launch_mix_dense_tc(const HopLaunchCfg& c, const void* mapX, const void*
     std::memcpy(&mg, mapG, sizeof(mg));
     std::memcpy(&my, mapY ? mapY : mapX, sizeof(my));
     const size_t smem = hop_dense_tc_smem(Kpad);
-    cudaError_t e = cudaFuncSetAttribute(mix_dense_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = hop_allow_max_smem<mix_dense_tc_kernel>();
     if (e != cudaSuccess) return (int)e;
     const int64_t tiles = c.P / kTile;
     const int grid = (int)std::min<int64_t>(tiles, (int64_t)c.sm_count);

@@ -88,6 +88,25 @@ void hop_build_level(const HopGraph& g, int32_t s, int32_t level, const int32_t*
                      const int32_t* nbr, const int32_t* ver, const int32_t* num, const int32_t* den,
                      HopLevelHost& out);
 
+// Opt a kernel into the largest dynamic shared-memory size once per device instead of before every launch
+// (the call is not a stream operation, so this also keeps it out of stream capture).
+#ifdef __CUDACC__
+template <auto Kernel>
+static inline cudaError_t hop_allow_max_smem() {
+    static bool done[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (!done[dev]) {
+        e = cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        done[dev] = true;
+    }
+    return cudaSuccess;
+}
+#endif
+
 // hop_kernels.cu : launchers.  All return a cudaError_t cast to int.
 struct HopLaunchCfg {
     float* X; float* M; float* G;

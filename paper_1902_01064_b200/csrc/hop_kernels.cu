@@ -397,7 +397,7 @@ int hop_launch_mix_staged(const HopLaunchCfg& c, const HopLevelDev& lv) {
     cudaError_t e = cudaSuccess;
 #define HOP_LAUNCH_STAGED(V, MO)                                                                              \
     do {                                                                                                      \
-        e = cudaFuncSetAttribute(mix_staged_kernel<V, MO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        e = hop_allow_max_smem<mix_staged_kernel<V, MO>>();                                                   \
         if (e == cudaSuccess)                                                                                 \
             mix_staged_kernel<V, MO><<<grid, kStagedThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, lv); \
     } while (0)
@@ -420,11 +420,11 @@ int hop_launch_mix_bulk(const HopLaunchCfg& c, const HopLevelDev& lv) {
     cudaStream_t st = (cudaStream_t)c.stream;
     cudaError_t e;
     if (c.mu != 0.f) {
-        e = cudaFuncSetAttribute(mix_bulk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e = hop_allow_max_smem<mix_bulk_kernel<true>>();
         if (e != cudaSuccess) return (int)e;
         mix_bulk_kernel<true><<<grid, kBulkThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, lv, c.table_smem, c.n_ents, c.err_word);
     } else {
-        e = cudaFuncSetAttribute(mix_bulk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e = hop_allow_max_smem<mix_bulk_kernel<false>>();
         if (e != cudaSuccess) return (int)e;
         mix_bulk_kernel<false><<<grid, kBulkThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, lv, c.table_smem, c.n_ents, c.err_word);
     }

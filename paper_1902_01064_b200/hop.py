@@ -21,7 +21,7 @@ W_UNIFORM, W_STALE_LINEAR = 0, 1
 GRAD_EXTERNAL, GRAD_SYNTHETIC, GRAD_SVM_DENSE, GRAD_SVM_CSR = 0, 1, 2, 3
 MIX_AUTO, MIX_STAGED, MIX_BULK, MIX_TENSOR = 0, 1, 2, 3
 (OPT_MAX_IG, OPT_LR, OPT_MOMENTUM, OPT_WEIGHT_MODE, OPT_GRAD_MODE, OPT_GRAD_SEED, OPT_GRAD_SIGMA,
- OPT_MIX_KERNEL, OPT_COL_OFFSET) = range(1, 10)
+ OPT_MIX_KERNEL, OPT_COL_OFFSET, OPT_USE_GRAPH) = range(1, 11)
 OPT_BACKUP_OF_WORKER = 1000
 
 _p = C.c_void_p
@@ -46,6 +46,7 @@ SIGNATURES = {
     "hop_newest_version": [_p, _i32, C.POINTER(_i32)],
     "hop_set_level": [_p, _i32],
     "hop_step": [_p],
+    "hop_run": [_p, _i32],
     "hop_step_host": [_p, _p, _p, _p, _p, _p, _p, _p, _i64],
     "hop_read_status": [_p, C.POINTER(_i32)],
     "hop_level_stats": [_p, _i32, _p],
@@ -179,6 +180,9 @@ class Hop:
 
     def step(self):
         self._chk(lib.hop_step(self.h))
+
+    def run(self, n_levels):
+        self._chk(lib.hop_run(self.h, n_levels))
 
     def step_host(self, op, ptr, nbr, ver, num, den, probe=None):
         """One level from host arrays (already contiguous int32/int64 numpy); probe: float32 numpy or None."""
