@@ -163,6 +163,8 @@ def main():
     ap.add_argument("--mix-kernel", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--graph", default="auto", choices=["auto", "0", "1"],
+                    help="timed region replays CUDA graphs of the trace (hop_run); auto = only for small, launch-bound workloads")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -194,7 +196,9 @@ def main():
     X = torch.zeros((w.N, S, w.P), dtype=torch.float32, device=dev)
     M = torch.zeros((w.N, w.P), dtype=torch.float32, device=dev) if w.momentum else None
     G = None if w.grad_mode == inputs.GRAD_SVM_CSR else torch.zeros((w.N, w.P), dtype=torch.float32, device=dev)
-    stream = torch.cuda.current_stream()
+    stream = torch.cuda.Stream(device=dev)      # a capturable stream; torch's own fills and copies follow it too
+    torch.cuda.set_stream(stream)
+    use_graph = args.graph == "1" or (args.graph == "auto" and X.numel() * 4 < 2e9)
     h = hop.from_workload(w, args.mix_kernel)
     h.set_option(hop.OPT_COL_OFFSET, lo)
     h.bind_buffers(X, M, G, stream.cuda_stream)
@@ -229,8 +233,9 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
-    def run_levels(n, first=0):
-        """n consecutive levels starting at trace level `first` (mod the trace length)."""
+    def run_levels(n, first=0, graph=False):
+        """n consecutive levels starting at trace level `first` (mod the trace length); with graph=True whole
+        stretches of the trace go through hop_run, which replays a cached CUDA graph."""
         done = 0
         k = first % w.iters
         h.set_level(k)
@@ -239,34 +244,46 @@ def main():
             if k == w.iters:
                 k = 0
                 h.set_level(0)
-            h.step()
-            wi += int(wi_per_level[k])
-            timed["flops"] += stats[k]["mma_flops"]
-            k += 1
-            done += 1
+            m = min(n - done, w.iters - k) if graph else 1
+            if graph:
+                h.run(m)
+            else:
+                h.step()
+            wi += int(wi_per_level[k:k + m].sum())
+            timed["flops"] += sum(st["mma_flops"] for st in stats[k:k + m])
+            k += m
+            done += m
         return wi
 
     # ---- warm-up, then the timed region: exactly K steps between two events on the launching stream
     reset()
     run_levels(max(3, args.warmup))
+    if use_graph:                      # instantiate the graphs outside the timed region
+        reset()
+        run_levels(args.steps, graph=True)
     reset()
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
     launches0 = h.launch_count()
-    h.timing_enable(True)
+    h.timing_enable(not use_graph)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     timed["flops"] = 0
-    wi = run_levels(args.steps)
+    wi = run_levels(args.steps, graph=use_graph)
     mma_flops = timed["flops"]
     e1.record(stream)
     barrier()
     sampler.stop_flag = True
     ms = e0.elapsed_time(e1)
+    launches = h.launch_count() - launches0
+    if use_graph:                      # per-kernel event timing is not possible inside a replayed graph: separate pass
+        reset()
+        h.timing_enable(True)
+        run_levels(args.steps)
+        torch.cuda.synchronize()
     tim = h.timing_read()
     h.timing_enable(False)
-    launches = h.launch_count() - launches0
     assert h.read_status() == 0
     sampler.join(timeout=1.0)
     if dist is not None:
@@ -325,6 +342,8 @@ def main():
     traffic = NCU_TRAFFIC.get((args.config, P_global))
     roofline = {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
                 "traffic": traffic, "traffic_unit": "bytes per launch", "peak_kind": f"of {peak_kind}", "kernel": "+".join(kname[k] for k in kernels),
+                "kernel_timing": ("separate step-by-step pass with per-kernel events (the timed region replays CUDA graphs)"
+                                  if use_graph else "CUDA events inside the timed region"),
                 "launches": mix_launches, "avg_launch_ms": tim["ms_mix"] / max(1, mix_launches),
                 "alg_bytes_per_launch": tim["mix_bytes"] / max(1, mix_launches),
                 "frac_of_nominal_8TBs": ach / 8000.0,
@@ -343,7 +362,8 @@ def main():
             "config": {"workload": f"config {args.config}: {w.name}", "N": w.N, "P": P_global, "P_per_gpu": w.P, "s": w.s, "b": w.b,
                        "levels": w.iters, "trace_passes": args.steps / w.iters, "parallelism": f"column-sharded x{world}",
                        "l2": "inputs exceed L2 (ring %.1f GB per GPU)" % (X.numel() * 4 / 1e9) if X.numel() * 4 > 3e8 else "ring fits L2: absolute numbers only",
-                       "protocol_sim_ms": sim_ms},
+                       "protocol_sim_ms": sim_ms,
+                       "launch": "hop_run: CUDA graph replay of the trace" if use_graph else "hop_step per level"},
             "roofline": roofline, "gpu_launches": int(launches), "clocks": sampler.result()}
     if e2e is not None:
         line["e2e"] = e2e
