@@ -67,6 +67,12 @@ typedef enum hop_op {
  * STALE_LINEAR: numerator Iter(u) - (k - s) + 1, normalised (Eq. 2). */
 typedef enum hop_weight_mode { HOP_W_UNIFORM = 0, HOP_W_STALE_LINEAR = 1 } hop_weight_mode;
 
+/* What Recv keeps once |N_in(i)| - N_buw(i) in-neighbours are usable.  AT_LEAST: every usable update
+ * (Fig. alg4: the needed ones, then "any additional update" in the queue).  EXACT: exactly
+ * |N_in(i)| - N_buw(i): the own update plus the neighbours whose first usable update was sent
+ * earliest (what a FIFO dequeue of that many entries returns), ties by worker id. */
+typedef enum hop_backup_mode { HOP_BACKUP_AT_LEAST = 0, HOP_BACKUP_EXACT = 1 } hop_backup_mode;
+
 /* Where the gradient of a level comes from. */
 typedef enum hop_grad_mode {
     HOP_GRAD_EXTERNAL = 0,   /* the caller fills G before each hop_step                            */
@@ -95,7 +101,8 @@ typedef enum hop_option {
     HOP_OPT_MIX_KERNEL = 8,   /* hop_mix_kernel (default AUTO)                                      */
     HOP_OPT_COL_OFFSET = 9,   /* global index of local parameter 0 when P is a shard of a larger    */
                               /* vector (multiple of 4); only the synthetic gradient reads it       */
-    HOP_OPT_USE_GRAPH = 10,   /* hop_run may replay a captured CUDA graph (default 1)                    */
+    HOP_OPT_USE_GRAPH = 10,   /* hop_run may replay a captured CUDA graph (default 1)               */
+    HOP_OPT_BACKUP_MODE = 11, /* hop_backup_mode (default AT_LEAST)                                 */
     HOP_OPT_BACKUP_OF_WORKER = 1000 /* key = 1000 + i sets N_buw(i) of one worker (Fig. alg4)       */
 } hop_option;
 

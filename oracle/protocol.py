@@ -32,6 +32,10 @@ Readings taken where the paper is silent (listed once more in the design notes):
       k-1, and Reduces (a JUMP record at level k-1), then moves k-k0 tokens each way and enters
       k.  Levels k0+1 .. k-2 are IDLE; its updates k0+1 .. k-1 are never sent.
   R6  A worker that applied its last iteration stops (no token acquire after it).
+  R7  backup_exact (off by default; the paper's Fig. alg4 takes "any additional update"): Recv completes at the
+      same moment as under R3 but keeps exactly |N_in(i)| - b_i updates: its own, plus those in-neighbours
+      whose first satisfactory update (iter in [k-s, k]) arrived earliest in UpdateQ(i) (FIFO order of
+      Fig. alg4's dequeue); the version taken from a kept neighbour is still its newest one with iter <= k.
 """
 from __future__ import annotations
 
@@ -89,7 +93,7 @@ def reduce_weights(vers, level, s, weight_mode):
 
 class HopProtocol:
     def __init__(self, n_in, ticks, iters, s=0, b=0, max_ig=None, max_skip=0,
-                 weight_mode=UNIFORM, on_round=None):
+                 weight_mode=UNIFORM, on_round=None, backup_exact=False):
         self.N = N = len(n_in)
         self.n_in = [list(nb) for nb in n_in]
         for i, nb in enumerate(self.n_in):
@@ -113,6 +117,9 @@ class HopProtocol:
         self.weight_mode = weight_mode
         self.on_round = on_round
         # ---- literal queues
+        self.backup_exact = backup_exact
+        self.arrivals = [0] * N                                # entries ever enqueued into UpdateQ(i)
+        self.arrival_pos = {}                                  # (w_id, i) -> {iter: position in UpdateQ(i)'s arrival order}
         self.update_q = [[] for _ in range(N)]                 # FIFO of (iter, w_id) tags
         self.iter_rcv = {(j, i): -1 for i in range(N) for j in self.n_in[i]}
         self.token_q = {}
@@ -137,6 +144,8 @@ class HopProtocol:
                     self.token_q[(i, j)].extend([k] * n_tokens)
         for j in self.n_out[i]:
             self.update_q[j].append((k, i))                     # UpdateQ(j).enqueue(x_{k,i}, iter=k, w_id=i)
+            self.arrival_pos.setdefault((i, j), {})[k] = self.arrivals[j]
+            self.arrivals[j] += 1
         self.Iter[i] = k
         self.phase[i] = _COMPUTE
         self.end[i] = self.now + int(self.ticks[i][k])
@@ -162,9 +171,17 @@ class HopProtocol:
                 got.append((j, own_version))                     # jumper's current parameters
             elif self.iter_rcv[(j, i)] >= level - self.s:
                 got.append((j, self.iter_rcv[(j, i)]))
-        if len(got) >= len(self.n_in[i]) - self.b[i]:
-            return got
-        return None
+        need = len(self.n_in[i]) - self.b[i]
+        if len(got) < need:
+            return None
+        if self.backup_exact and len(got) > need:
+            def first_satisfactory_arrival(j):
+                seen = self.arrival_pos[(j, i)]
+                return min(seen[it] for it in range(level - self.s, level + 1) if it in seen)
+            others = sorted((jv for jv in got if jv[0] != i), key=lambda jv: (first_satisfactory_arrival(jv[0]), jv[0]))
+            keep = {i} | {j for j, _ in others[:need - 1]}
+            got = [jv for jv in got if jv[0] in keep]
+        return got
 
     def _record(self, op, level, i, got, own_as=None):
         vers = [(own_as if (j == i and own_as is not None) else v) for (j, v) in got]
@@ -254,8 +271,9 @@ class HopProtocol:
         return self.trace
 
 
-def simulate(n_in, ticks, iters, s=0, b=0, max_ig=None, max_skip=0, weight_mode=UNIFORM, on_round=None):
-    return HopProtocol(n_in, ticks, iters, s, b, max_ig, max_skip, weight_mode, on_round).run()
+def simulate(n_in, ticks, iters, s=0, b=0, max_ig=None, max_skip=0, weight_mode=UNIFORM, on_round=None,
+             backup_exact=False):
+    return HopProtocol(n_in, ticks, iters, s, b, max_ig, max_skip, weight_mode, on_round, backup_exact).run()
 
 
 # -------------------------------------------------------------------- graph helpers for the invariants

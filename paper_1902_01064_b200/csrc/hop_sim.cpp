@@ -42,6 +42,8 @@ struct Sim {
     std::vector<Phase> phase;
     std::vector<int32_t> jump_to;
     std::vector<std::vector<int32_t>> entered;      // iterations a worker has entered, ascending
+    std::vector<std::vector<int64_t>> entered_seq;  // global order of those Send events (arrival order at every receiver)
+    int64_t send_seq = 0;
     uint64_t now = 0;
     using Ev = std::pair<uint64_t, int32_t>;
     std::priority_queue<Ev, std::vector<Ev>, std::greater<Ev>> compute_end;
@@ -51,7 +53,7 @@ struct Sim {
 
     Sim(const HopGraph& g_, const HopSimParams& p_, const uint64_t* t, int32_t it, hop_trace& o)
         : g(g_), p(p_), ticks(t), iters(it), N(g_.N), iter(N, 0), phase(N, COMPUTE), jump_to(N, 0),
-          entered(N), r_nbr((size_t)it * N), r_ver((size_t)it * N), r_num((size_t)it * N), out(o) {}
+          entered(N), entered_seq(N), r_nbr((size_t)it * N), r_ver((size_t)it * N), r_num((size_t)it * N), out(o) {}
 
     int32_t newest_entered_upto(int32_t j, int32_t level) const {
         const auto& e = entered[j];
@@ -62,6 +64,7 @@ struct Sim {
     void enter(int32_t i, int32_t k) {
         iter[i] = k;
         entered[i].push_back(k);
+        entered_seq[i].push_back(send_seq++);
         phase[i] = COMPUTE;
         compute_end.push({now + ticks[(size_t)i * iters + k], i});
     }
@@ -75,7 +78,27 @@ struct Sim {
             const int32_t v = newest_entered_upto(j, level);
             if (v >= 0 && v >= level - p.s) d.got.push_back({j, v});
         }
-        return (int32_t)d.got.size() >= (e - a) - p.b[i];
+        const int32_t need = (e - a) - p.b[i];
+        if ((int32_t)d.got.size() < need) return false;
+        if (p.backup_exact && (int32_t)d.got.size() > need) {
+            // keep the own update plus the neighbours whose first usable update (iteration >= level - s) was sent
+            // earliest: the first |N_in| - b entries a FIFO dequeue would return
+            std::vector<std::pair<int64_t, int32_t>> order;   // (send order of first usable update, neighbour)
+            for (auto [j, v] : d.got) {
+                if (j == i) continue;
+                const auto& en = entered[j];
+                const size_t pos = std::lower_bound(en.begin(), en.end(), std::max(0, level - p.s)) - en.begin();
+                order.push_back({entered_seq[j][pos], j});
+            }
+            std::sort(order.begin(), order.end());
+            std::vector<uint8_t> keep(N, 0);
+            keep[i] = 1;
+            for (int32_t t = 0; t < need - 1; ++t) keep[order[t].second] = 1;
+            std::vector<std::pair<int32_t, int32_t>> kept;
+            for (auto jv : d.got) if (keep[jv.first]) kept.push_back(jv);
+            d.got.swap(kept);
+        }
+        return true;
     }
 
     Decision decide(int32_t i) const {

@@ -358,3 +358,19 @@ def test_deadlock_is_reported():
             return False
     with pytest.raises(op.Deadlock):
         NoTokens(inputs.ring(4), np.ones((4, 3), np.uint64), 3, max_ig=1).run()
+
+
+def test_exact_backup_keeps_own_update_and_earliest_senders():
+    # worker 0 listens to 1, 2, 3 (and itself), b = 2: it keeps its own update and ONE neighbour, the one whose
+    # update of the iteration arrived first in its queue.  Senders enter iteration 1 at ticks 2, 5, 3.
+    n_in = [[0, 1, 2, 3], [1], [2], [3]]
+    ticks = np.array([[9, 1], [2, 1], [5, 1], [3, 1]], np.uint64)
+    tr = op.simulate(n_in, ticks, 2, s=0, b=[2, 0, 0, 0], max_ig=None, backup_exact=True)
+    assert [(j, v) for j, v, _ in tr.rec[(0, 0)]] == [(0, 0), (1, 0)]           # all sent iteration 0 at tick 0: ties by id
+    assert [(j, v) for j, v, _ in tr.rec[(1, 0)]] == [(0, 1), (1, 1)]           # worker 1 entered iteration 1 first
+    assert tr.den[(1, 0)] == 2
+    loose = op.simulate(n_in, ticks, 2, s=0, b=[2, 0, 0, 0], max_ig=None)
+    assert [j for j, _, _ in loose.rec[(1, 0)]] == [0, 1, 2, 3]                 # Fig. alg4 takes every available one
+    # with staleness the kept neighbour's *newest* update is consumed, but the order is that of the first usable one
+    tr = op.simulate(n_in, np.array([[9, 9], [2, 1], [1, 30], [3, 1]], np.uint64), 2, s=1, b=[2, 0, 0, 0], max_ig=None, backup_exact=True)
+    assert [(j, v) for j, v, _ in tr.rec[(1, 0)]] == [(0, 1), (1, 1)]

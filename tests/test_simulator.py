@@ -11,14 +11,15 @@ from paper_1902_01064_b200 import hop, inputs
 KEYS = ("op", "ptr", "nbr", "ver", "num", "den")
 
 
-def both(n_in, ticks, iters, s, b, max_ig, max_skip, mode):
+def both(n_in, ticks, iters, s, b, max_ig, max_skip, mode, exact=False):
     ptr, idx = inputs.graph_to_csr(n_in)
     n_in = inputs.csr_to_lists(ptr, idx)                 # records list neighbours in ascending id order
     h = hop.Hop(ptr, idx, len(n_in), 8, s, b, max_skip)
     h.set_option(hop.OPT_MAX_IG, 0 if max_ig is None else max_ig)
     h.set_option(hop.OPT_WEIGHT_MODE, mode)
+    h.set_option(hop.OPT_BACKUP_MODE, hop.BACKUP_EXACT if exact else hop.BACKUP_AT_LEAST)
     got = h.sim_run(ticks, iters).to_arrays()
-    want_tr = op.simulate(n_in, ticks, iters, s, b, max_ig, max_skip, mode)
+    want_tr = op.simulate(n_in, ticks, iters, s, b, max_ig, max_skip, mode, backup_exact=exact)
     want = want_tr.to_arrays()
     h.close()
     return got, want, want_tr.makespan
@@ -112,3 +113,45 @@ def test_unbounded_gap_without_tokens():
     ticks[0, 0] = 10 ** 12
     got, want, mk = both(n_in, ticks, 12, 0, 1, None, 0, op.UNIFORM)
     assert_same(got, want, mk)
+
+
+def test_exact_backup_mode_bit_exact_and_exactly_d_minus_b():
+    rng = np.random.default_rng(77)
+    for trial in range(40):
+        N = int(rng.integers(4, 12))
+        n_in = [{i, (i - 1) % N, (i + 1) % N} for i in range(N)]
+        for _ in range(int(rng.integers(N, 4 * N))):
+            a, c = rng.integers(0, N, 2)
+            n_in[int(a)].add(int(c))
+        n_in = [sorted(x) for x in n_in]
+        s = int(rng.integers(0, 3))
+        b = int(rng.integers(1, min(len(x) for x in n_in)))
+        max_skip = int(rng.integers(0, s + 2)) if trial % 2 else 0
+        iters = 20
+        ticks = rng.choice([1, 2, 3, 9], size=(N, iters)).astype(np.uint64)
+        try:
+            got, want, mk = both(n_in, ticks, iters, s, b, 3, max_skip, op.STALE_LINEAR, exact=True)
+        except op.Deadlock:
+            continue
+        assert_same(got, want, mk, trial)
+        cnt = np.diff(got["ptr"]).reshape(iters, N)
+        for i in range(N):
+            active = got["op"][:, i] != op.IDLE
+            assert (cnt[active, i] == len(n_in[i]) - b).all()          # exactly in-degree - b consumed
+    for name, n_in in inputs.small_cases():
+        if name.endswith("3"):
+            continue
+        for flat in itertools.product((1, 2, 3), repeat=8):
+            ticks = np.asarray(flat, np.uint64).reshape(4, 2)
+            got, want, mk = both(n_in, ticks, 2, 1, 1, 1, 0, op.UNIFORM, exact=True)
+            assert_same(got, want, mk, (name, flat))
+
+
+@pytest.mark.parametrize("cfg", [2, 4, 5])
+def test_configs_bit_exact_in_exact_backup_mode(cfg):
+    w = inputs.make_workload(cfg, P=256)
+    got, want, mk = both(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode, exact=True)
+    assert_same(got, want, mk, cfg)
+    d = np.diff(w.in_ptr)
+    cnt = np.diff(got["ptr"]).reshape(w.iters, w.N)
+    assert (cnt == (d - w.b)[None, :]).all()
