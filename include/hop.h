@@ -103,6 +103,9 @@ typedef enum hop_option {
                               /* vector (multiple of 4); only the synthetic gradient reads it       */
     HOP_OPT_USE_GRAPH = 10,   /* hop_run may replay a captured CUDA graph (default 1)               */
     HOP_OPT_BACKUP_MODE = 11, /* hop_backup_mode (default AT_LEAST)                                 */
+    HOP_OPT_NOTIFY_ACK = 12,  /* 1: simulate the NOTIFY-ACK scheme of Section 3.3 (the paper's baseline)  */
+                              /* instead of token queues: iteration k+1 is entered only once every   */
+                              /* out-neighbour has reduced iteration k-1; max_ig is ignored          */
     HOP_OPT_BACKUP_OF_WORKER = 1000 /* key = 1000 + i sets N_buw(i) of one worker (Fig. alg4)       */
 } hop_option;
 

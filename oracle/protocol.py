@@ -32,6 +32,12 @@ Readings taken where the paper is silent (listed once more in the design notes):
       k-1, and Reduces (a JUMP record at level k-1), then moves k-k0 tokens each way and enters
       k.  Levels k0+1 .. k-2 are IDLE; its updates k0+1 .. k-1 are never sent.
   R6  A worker that applied its last iteration stops (no token acquire after it).
+  R8  notify_ack=True replaces the token queues by the NOTIFY-ACK scheme of Section 3.3 (prior work, the paper's
+      baseline): after the Reduce of iteration k a worker sends ACK(k) to its in-neighbours, and a worker enters
+      iteration k+1 only with ACK(k-1) from every out-neighbour.  That is the reading that reproduces the bounds
+      the paper states for it (Table 1: a receiver at most 1 ahead of its sender, a sender at most 2 ahead of its
+      receiver) and the Section 3.4 example (B and C stuck in iteration 1 waiting for ACK(0)); the Section 3.5
+      remark that they could not even enter iteration 1 is at odds with both and is not followed.
   R7  backup_exact (off by default; the paper's Fig. alg4 takes "any additional update"): Recv completes at the
       same moment as under R3 but keeps exactly |N_in(i)| - b_i updates: its own, plus those in-neighbours
       whose first satisfactory update (iter in [k-s, k]) arrived earliest in UpdateQ(i) (FIFO order of
@@ -93,7 +99,7 @@ def reduce_weights(vers, level, s, weight_mode):
 
 class HopProtocol:
     def __init__(self, n_in, ticks, iters, s=0, b=0, max_ig=None, max_skip=0,
-                 weight_mode=UNIFORM, on_round=None, backup_exact=False):
+                 weight_mode=UNIFORM, on_round=None, backup_exact=False, notify_ack=False):
         self.N = N = len(n_in)
         self.n_in = [list(nb) for nb in n_in]
         for i, nb in enumerate(self.n_in):
@@ -117,6 +123,10 @@ class HopProtocol:
         self.weight_mode = weight_mode
         self.on_round = on_round
         # ---- literal queues
+        self.notify_ack = notify_ack
+        if notify_ack and (max_ig is not None or max_skip > 0):
+            raise ValueError("NOTIFY-ACK replaces the token queues (max_ig=None) and has no skipping")
+        self.acks = {(j, i): [] for i in range(N) for j in self.n_out[i] if j != i}   # ACKs from j received at i
         self.backup_exact = backup_exact
         self.arrivals = [0] * N                                # entries ever enqueued into UpdateQ(i)
         self.arrival_pos = {}                                  # (w_id, i) -> {iter: position in UpdateQ(i)'s arrival order}
@@ -191,6 +201,9 @@ class HopProtocol:
         self.trace.den[(level, i)] = den
 
     def _tokens_available(self, i, n):
+        if self.notify_ack:                                       # ACK(k-1) from every out-neighbour
+            k = self.Iter[i]
+            return k - 1 < 0 or all((k - 1) in self.acks[(j, i)] for j in self.n_out[i] if j != i)
         if self.max_ig is None:
             return True
         return all(len(self.token_q[(j, i)]) >= n for j in self.n_out[i] if j != i)
@@ -232,6 +245,10 @@ class HopProtocol:
         k = self.Iter[i]
         if act[0] == "applied":
             self._record(NORMAL, k, i, act[1])
+            if self.notify_ack:
+                for j in self.n_in[i]:
+                    if j != i:
+                        self.acks[(i, j)].append(k)              # ACK(k) after the Reduce, to every in-neighbour
             self.phase[i] = _DONE if k == self.iters - 1 else _TOKEN
         elif act[0] == "enter":
             self._take_tokens(i, 1)
@@ -272,8 +289,8 @@ class HopProtocol:
 
 
 def simulate(n_in, ticks, iters, s=0, b=0, max_ig=None, max_skip=0, weight_mode=UNIFORM, on_round=None,
-             backup_exact=False):
-    return HopProtocol(n_in, ticks, iters, s, b, max_ig, max_skip, weight_mode, on_round, backup_exact).run()
+             backup_exact=False, notify_ack=False):
+    return HopProtocol(n_in, ticks, iters, s, b, max_ig, max_skip, weight_mode, on_round, backup_exact, notify_ack).run()
 
 
 # -------------------------------------------------------------------- graph helpers for the invariants

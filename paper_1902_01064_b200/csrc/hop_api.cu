@@ -154,6 +154,7 @@ extern "C" int hop_set_option(hop_ctx* c, int key, double v) {
     if (!c) return HOP_E_ARG;
     drop_graphs(c);
     if (key == HOP_OPT_USE_GRAPH) { c->use_graph = v != 0.0; return HOP_OK; }
+    if (key == HOP_OPT_NOTIFY_ACK) { c->sp.notify_ack = v != 0.0; return HOP_OK; }
     if (key == HOP_OPT_BACKUP_MODE) {
         if (v != HOP_BACKUP_AT_LEAST && v != HOP_BACKUP_EXACT) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: unknown backup mode");
         c->sp.backup_exact = (int32_t)v;

@@ -73,6 +73,7 @@ struct HopGraph {
 
 struct HopSimParams {
     int32_t s, max_ig /*0 = none*/, max_skip, weight_mode;
+    int32_t notify_ack = 0;     // NOTIFY-ACK back-pressure (Section 3.3) instead of token queues
     int32_t backup_exact = 0;   // keep exactly |N_in| - b updates (own + earliest senders) instead of every usable one
     std::vector<int32_t> b;
 };

@@ -41,6 +41,7 @@ struct Sim {
     std::vector<int32_t> iter;                      // iteration a worker is in
     std::vector<Phase> phase;
     std::vector<int32_t> jump_to;
+    std::vector<int32_t> applied;                   // newest iteration whose Reduce/Apply is done (-1: none)
     std::vector<std::vector<int32_t>> entered;      // iterations a worker has entered, ascending
     std::vector<std::vector<int64_t>> entered_seq;  // global order of those Send events (arrival order at every receiver)
     int64_t send_seq = 0;
@@ -52,7 +53,7 @@ struct Sim {
     hop_trace& out;
 
     Sim(const HopGraph& g_, const HopSimParams& p_, const uint64_t* t, int32_t it, hop_trace& o)
-        : g(g_), p(p_), ticks(t), iters(it), N(g_.N), iter(N, 0), phase(N, COMPUTE), jump_to(N, 0),
+        : g(g_), p(p_), ticks(t), iters(it), N(g_.N), iter(N, 0), phase(N, COMPUTE), jump_to(N, 0), applied(N, -1),
           entered(N), entered_seq(N), r_nbr((size_t)it * N), r_ver((size_t)it * N), r_num((size_t)it * N), out(o) {}
 
     int32_t newest_entered_upto(int32_t j, int32_t level) const {
@@ -109,13 +110,18 @@ struct Sim {
             if (try_recv(i, k, -1, d)) d.kind = Decision::APPLIED;
             break;
         case WAIT_TOKEN: {
-            int32_t slowest = INT32_MAX;
+            int32_t slowest = INT32_MAX, least_applied = INT32_MAX;
             bool any = false;
             for (int32_t t = g.out_ptr[i]; t < g.out_ptr[i + 1]; ++t) {
                 const int32_t j = g.out_idx[t];
                 if (j == i) continue;
                 any = true;
                 slowest = std::min(slowest, iter[j]);
+                least_applied = std::min(least_applied, applied[j]);
+            }
+            if (p.notify_ack) {   // NOTIFY-ACK: every out-neighbour has acknowledged (reduced) iteration k-1
+                if (!any || least_applied >= k - 1) { d.kind = Decision::ENTER; d.target = k + 1; }
+                break;
             }
             if (p.max_skip > 0 && any) {
                 const int32_t behind = slowest - (k + 1);
@@ -189,6 +195,8 @@ struct Sim {
                     switch (d.kind) {
                     case Decision::APPLIED:
                         record(HOP_OP_NORMAL, k, i, d, -1);
+                        applied[i] = k;
+                        if (p.notify_ack) touch_neighbours(i, next_dirty);   // an ACK may release an in-neighbour
                         if (k == iters - 1) { phase[i] = DONE; ++done; } else phase[i] = WAIT_TOKEN;
                         break;
                     case Decision::ENTER:
@@ -228,6 +236,7 @@ int hop_simulate(const HopGraph& g, const HopSimParams& p, const uint64_t* ticks
                  hop_trace& out, std::string& err) {
     for (size_t t = 0; t < (size_t)g.N * iters; ++t)
         if (ticks[t] == 0) { err = "compute time of 0 ticks"; return HOP_E_ARG; }
+    if (p.notify_ack && p.max_skip > 0) { err = "NOTIFY-ACK has no iteration skipping"; return HOP_E_ARG; }
     if (p.max_skip > 0 && p.max_ig == 0) { err = "skipping reads token counts: token queues (max_ig >= 1) required"; return HOP_E_ARG; }
     Sim sim(g, p, ticks, iters, out);
     return sim.run(err);

@@ -21,7 +21,7 @@ W_UNIFORM, W_STALE_LINEAR = 0, 1
 GRAD_EXTERNAL, GRAD_SYNTHETIC, GRAD_SVM_DENSE, GRAD_SVM_CSR = 0, 1, 2, 3
 MIX_AUTO, MIX_STAGED, MIX_BULK, MIX_TENSOR = 0, 1, 2, 3
 (OPT_MAX_IG, OPT_LR, OPT_MOMENTUM, OPT_WEIGHT_MODE, OPT_GRAD_MODE, OPT_GRAD_SEED, OPT_GRAD_SIGMA,
- OPT_MIX_KERNEL, OPT_COL_OFFSET, OPT_USE_GRAPH, OPT_BACKUP_MODE) = range(1, 12)
+ OPT_MIX_KERNEL, OPT_COL_OFFSET, OPT_USE_GRAPH, OPT_BACKUP_MODE, OPT_NOTIFY_ACK) = range(1, 13)
 BACKUP_AT_LEAST, BACKUP_EXACT = 0, 1
 OPT_BACKUP_OF_WORKER = 1000
 

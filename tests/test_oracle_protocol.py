@@ -374,3 +374,43 @@ def test_exact_backup_keeps_own_update_and_earliest_senders():
     # with staleness the kept neighbour's *newest* update is consumed, but the order is that of the first usable one
     tr = op.simulate(n_in, np.array([[9, 9], [2, 1], [1, 30], [3, 1]], np.uint64), 2, s=1, b=[2, 0, 0, 0], max_ig=None, backup_exact=True)
     assert [(j, v) for j, v, _ in tr.rec[(1, 0)]] == [(0, 1), (1, 1)]
+
+
+@pytest.mark.parametrize("name,n_in", GRAPHS)
+def test_notify_ack_gap_bounds_of_table1(name, n_in):
+    # Table 1, row "Using NOTIFY-ACK": 1 towards in-neighbours, 2 towards out-neighbours,
+    # min(dist(j->i), 2 dist(i->j)) for arbitrary pairs
+    rng = np.random.default_rng(21)
+    N = len(n_in)
+    dist = op.shortest_paths(n_in)
+    worst = [0]
+    for trial in range(8):
+        def chk(p):
+            for i in range(N):
+                for j in range(N):
+                    if i != j:
+                        assert p.Iter[i] - p.Iter[j] <= min(dist[j][i], 2 * dist[i][j])
+                        if dist[i][j] == 1:
+                            worst[0] = max(worst[0], p.Iter[i] - p.Iter[j])
+        op.simulate(n_in, rand_ticks(rng, N, 12, 1, 30), 12, notify_ack=True, on_round=chk)
+    if name == "cycle5":
+        assert worst[0] == 2                                        # the bound of 2 is reached on a one-way edge
+
+
+def test_notify_ack_prose_example_and_no_room_for_backup_workers():
+    # Section 3.4: with NOTIFY-ACK, B and C are stuck in iteration 1 waiting for ACK(0) from A even though one
+    # update would do (backup workers); with token queues they advance to max_ig.
+    n_in = inputs.complete(3)
+    ticks = np.ones((3, 10), np.uint64)
+    ticks[0, 0] = STUCK
+    top = [0, 0, 0]
+
+    def chk(p):
+        if p.now < STUCK:
+            for i in range(3):
+                top[i] = max(top[i], p.Iter[i])
+    op.simulate(n_in, ticks, 10, s=0, b=1, notify_ack=True, on_round=chk)
+    assert top == [0, 1, 1]
+    top[:] = [0, 0, 0]
+    op.simulate(n_in, ticks, 10, s=0, b=1, max_ig=4, on_round=chk)
+    assert top == [0, 4, 4]

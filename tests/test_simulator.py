@@ -11,15 +11,17 @@ from paper_1902_01064_b200 import hop, inputs
 KEYS = ("op", "ptr", "nbr", "ver", "num", "den")
 
 
-def both(n_in, ticks, iters, s, b, max_ig, max_skip, mode, exact=False):
+def both(n_in, ticks, iters, s, b, max_ig, max_skip, mode, exact=False, notify_ack=False):
     ptr, idx = inputs.graph_to_csr(n_in)
     n_in = inputs.csr_to_lists(ptr, idx)                 # records list neighbours in ascending id order
     h = hop.Hop(ptr, idx, len(n_in), 8, s, b, max_skip)
     h.set_option(hop.OPT_MAX_IG, 0 if max_ig is None else max_ig)
     h.set_option(hop.OPT_WEIGHT_MODE, mode)
     h.set_option(hop.OPT_BACKUP_MODE, hop.BACKUP_EXACT if exact else hop.BACKUP_AT_LEAST)
+    h.set_option(hop.OPT_NOTIFY_ACK, 1 if notify_ack else 0)
     got = h.sim_run(ticks, iters).to_arrays()
-    want_tr = op.simulate(n_in, ticks, iters, s, b, max_ig, max_skip, mode, backup_exact=exact)
+    want_tr = op.simulate(n_in, ticks, iters, s, b, None if notify_ack else max_ig, max_skip, mode, backup_exact=exact,
+                          notify_ack=notify_ack)
     want = want_tr.to_arrays()
     h.close()
     return got, want, want_tr.makespan
@@ -155,3 +157,23 @@ def test_configs_bit_exact_in_exact_backup_mode(cfg):
     d = np.diff(w.in_ptr)
     cnt = np.diff(got["ptr"]).reshape(w.iters, w.N)
     assert (cnt == (d - w.b)[None, :]).all()
+
+
+def test_notify_ack_bit_exact():
+    rng = np.random.default_rng(5)
+    for trial in range(30):
+        N = int(rng.integers(3, 10))
+        n_in = [{i, (i - 1) % N} for i in range(N)]
+        for _ in range(int(rng.integers(0, 3 * N))):
+            a, c = rng.integers(0, N, 2)
+            n_in[int(a)].add(int(c))
+        n_in = [sorted(x) for x in n_in]
+        s = int(rng.integers(0, 3))
+        b = int(rng.integers(0, min(len(x) for x in n_in)))
+        ticks = rng.choice([1, 1, 2, 6], size=(N, 15)).astype(np.uint64)
+        got, want, mk = both(n_in, ticks, 15, s, b, 1, 0, op.UNIFORM, notify_ack=True)
+        assert_same(got, want, mk, trial)
+    for name, n_in in inputs.small_cases()[:2]:
+        for flat in itertools.product((1, 2, 3), repeat=9):
+            got, want, mk = both(n_in, np.asarray(flat, np.uint64).reshape(3, 3), 3, 0, 0, 1, 0, op.UNIFORM, notify_ack=True)
+            assert_same(got, want, mk, (name, flat))
