@@ -73,6 +73,15 @@ typedef enum hop_weight_mode { HOP_W_UNIFORM = 0, HOP_W_STALE_LINEAR = 1 } hop_w
  * earliest (what a FIFO dequeue of that many entries returns), ties by worker id. */
 typedef enum hop_backup_mode { HOP_BACKUP_AT_LEAST = 0, HOP_BACKUP_EXACT = 1 } hop_backup_mode;
 
+/* Loss of the linear model in the SVM modes: coef_r = d loss / d margin_r.
+ * HINGE: -y_r/B if y_r * margin_r < 1 else 0.   LOG: -y_r / (B * (1 + exp(y_r * margin_r))). */
+typedef enum hop_loss { HOP_LOSS_HINGE = 0, HOP_LOSS_LOG = 1 } hop_loss;
+
+/* Order of the five operations inside an iteration (Section 3.2).  PARALLEL: Send x_k, Compute on x_k, Recv,
+ * Reduce, Apply: x_{k+1} = Reduce(versions) - eta * d.  SERIAL: Compute, Apply, Send, Recv, Reduce:
+ * x'_k = x_k - eta * d replaces version k in the ring before anyone consumes it, x_{k+1} = Reduce(versions). */
+typedef enum hop_approach { HOP_APPROACH_PARALLEL = 0, HOP_APPROACH_SERIAL = 1 } hop_approach;
+
 /* Where the gradient of a level comes from. */
 typedef enum hop_grad_mode {
     HOP_GRAD_EXTERNAL = 0,   /* the caller fills G before each hop_step                            */
@@ -106,6 +115,9 @@ typedef enum hop_option {
     HOP_OPT_NOTIFY_ACK = 12,  /* 1: simulate the NOTIFY-ACK scheme of Section 3.3 (the paper's baseline)  */
                               /* instead of token queues: iteration k+1 is entered only once every   */
                               /* out-neighbour has reduced iteration k-1; max_ig is ignored          */
+    HOP_OPT_WEIGHT_DECAY = 13,/* lambda >= 0: lambda * x_{k,i} is added to the gradient (Section 7.2 uses 1e-4 / 1e-7)  */
+    HOP_OPT_LOSS = 14,        /* hop_loss of the SVM modes (default HINGE; the paper's runs used LOG, Section 7.2)    */
+    HOP_OPT_APPROACH = 15,    /* hop_approach (default PARALLEL, the paper's choice, Section 3.2)                     */
     HOP_OPT_BACKUP_OF_WORKER = 1000 /* key = 1000 + i sets N_buw(i) of one worker (Fig. alg4)       */
 } hop_option;
 

@@ -7,6 +7,9 @@ Train(), Reduce of Fig. alg4 or Eq. 2):
         d = g_{k,i}                      plain SGD (Fig. alg0: gradient of the pre-Reduce parameters,
                                          the "parallel approach" of Section 3.2)
         d = m <- mu*m + g_{k,i}          momentum; the buffer m is local and never averaged
+    weight decay lambda adds lambda * x_{k,i} to g (the experiments' regulariser, Section 7.2).
+    Serial approach (Section 3.2): Compute, Apply, then Send: x'_{k,i} = x_{k,i} - lr * d is what the worker sends
+    (it replaces version k), and x_{k+1,i} = sum (num/den) x'_{v,j}; all Applies of a level precede its Reduces.
     JUMP at level k (Section 5):  x_{k+1,i} = sum (num/den) x_{v,j}, no gradient; the worker's own
                                   entry names the version it actually holds.
     IDLE: nothing.
@@ -30,15 +33,25 @@ def hinge_coefficients(margins: np.ndarray, y: np.ndarray) -> np.ndarray:
     return np.where(y * margins < 1.0, -y / B, 0.0)
 
 
-def svm_gradient_dense(A: np.ndarray, y: np.ndarray, x: np.ndarray) -> np.ndarray:
-    """Sub-gradient of the mean hinge loss of a linear SVM (no bias, no regulariser) at x."""
+def log_coefficients(margins: np.ndarray, y: np.ndarray) -> np.ndarray:
+    """d/d(margin) of the mean log loss (1/B) sum_r log(1 + exp(-y_r m_r)) (the loss of the paper's SVM runs)."""
+    B = len(y)
+    return -y / (B * (1.0 + np.exp(y * margins)))
+
+
+def loss_coefficients(margins, y, loss="hinge"):
+    return hinge_coefficients(margins, y) if loss == "hinge" else log_coefficients(margins, y)
+
+
+def svm_gradient_dense(A: np.ndarray, y: np.ndarray, x: np.ndarray, loss="hinge") -> np.ndarray:
+    """(Sub-)gradient of the mean hinge or log loss of a linear model (no bias, no regulariser) at x."""
     A = A.astype(np.float64)
     y = y.astype(np.float64)
-    coef = hinge_coefficients(A @ x, y)
+    coef = loss_coefficients(A @ x, y, loss)
     return A.T @ coef
 
 
-def svm_gradient_csr(row_ptr, col, val, y, x: np.ndarray):
+def svm_gradient_csr(row_ptr, col, val, y, x: np.ndarray, loss="hinge"):
     """Same for CSR rows; returns (coef per row, dense gradient)."""
     y = y.astype(np.float64)
     B = len(y)
@@ -46,7 +59,7 @@ def svm_gradient_csr(row_ptr, col, val, y, x: np.ndarray):
     for r in range(B):
         a, e = row_ptr[r], row_ptr[r + 1]
         margins[r] = np.dot(val[a:e].astype(np.float64), x[col[a:e]])
-    coef = hinge_coefficients(margins, y)
+    coef = loss_coefficients(margins, y, loss)
     g = np.zeros_like(x)
     for r in range(B):
         if coef[r] != 0.0:
@@ -59,6 +72,10 @@ def mean_hinge_loss(A, y, x):
     return np.maximum(0.0, 1.0 - y.astype(np.float64) * (A.astype(np.float64) @ x)).mean()
 
 
+def mean_log_loss(A, y, x):
+    return np.logaddexp(0.0, -y.astype(np.float64) * (A.astype(np.float64) @ x)).mean()
+
+
 class GradSynthetic:
     def __init__(self, seed, sigma, cols):
         self.seed, self.sigma, self.cols = seed, sigma, np.asarray(cols, np.int64)
@@ -69,25 +86,25 @@ class GradSynthetic:
 
 class GradSvmDense:
     """Minibatch of iteration k = rows [(k mod R/B)*B, +B) of the worker's shard."""
-    def __init__(self, A, y, batch):
-        self.A, self.y, self.B = A, y, batch
+    def __init__(self, A, y, batch, loss="hinge"):
+        self.A, self.y, self.B, self.loss = A, y, batch, loss
 
     def __call__(self, k, i, x):
         R = self.A.shape[1]
         r0 = (k % (R // self.B)) * self.B
-        return svm_gradient_dense(self.A[i, r0:r0 + self.B], self.y[i, r0:r0 + self.B], x)
+        return svm_gradient_dense(self.A[i, r0:r0 + self.B], self.y[i, r0:r0 + self.B], x, self.loss)
 
 
 class GradSvmCsr:
-    def __init__(self, row_ptr, col, val, y, rows_per_worker, batch):
+    def __init__(self, row_ptr, col, val, y, rows_per_worker, batch, loss="hinge"):
         self.row_ptr, self.col, self.val, self.y = row_ptr, col, val, y
-        self.R, self.B = rows_per_worker, batch
+        self.R, self.B, self.loss = rows_per_worker, batch, loss
 
     def __call__(self, k, i, x):
         r0 = i * self.R + (k % (self.R // self.B)) * self.B
         rp = self.row_ptr[r0:r0 + self.B + 1]
         yy = self.y[i, (r0 - i * self.R):(r0 - i * self.R) + self.B]
-        _, g = svm_gradient_csr(rp, self.col, self.val, yy, x)
+        _, g = svm_gradient_csr(rp, self.col, self.val, yy, x, self.loss)
         return g
 
 
@@ -101,7 +118,7 @@ class GradExternal:
 
 
 def run_updates(tr: dict, N: int, lr: float, momentum: float, x0: np.ndarray, grad_fn,
-                levels=None, keep_all=False, s=None):
+                levels=None, keep_all=False, s=None, weight_decay=0.0, serial=False):
     """Execute levels 0..levels-1 of the trace arrays `tr` (see Trace.to_arrays).
 
     x0: [N][C] float64, version 0 of every worker.  Returns (X, newest) where X maps
@@ -111,7 +128,20 @@ def run_updates(tr: dict, N: int, lr: float, momentum: float, x0: np.ndarray, gr
     X = {(i, 0): np.array(x0[i], np.float64) for i in range(N)}
     newest = [0] * N
     M = [np.zeros(x0.shape[1]) for _ in range(N)] if momentum != 0.0 else None
+    def direction(k, i):
+        g = grad_fn(k, i, X[(i, k)])
+        if weight_decay != 0.0:
+            g = g + weight_decay * X[(i, k)]
+        if M is not None:
+            M[i] = momentum * M[i] + g
+            g = M[i]
+        return g
+
     for k in range(L):
+        if serial:                                   # Compute -> Apply -> Send: version k becomes x' before any Reduce
+            applied = {i: X[(i, k)] - lr * direction(k, i) for i in range(N) if op[k, i] == NORMAL}
+            for i, x in applied.items():
+                X[(i, k)] = x
         new = {}
         for i in range(N):
             o = op[k, i]
@@ -121,12 +151,8 @@ def run_updates(tr: dict, N: int, lr: float, momentum: float, x0: np.ndarray, gr
             mix = np.zeros(x0.shape[1])
             for t in range(a, e):
                 mix += (float(num[t]) / float(den[k, i])) * X[(int(nbr[t]), int(ver[t]))]
-            if o == NORMAL:
-                g = grad_fn(k, i, X[(i, k)])
-                if M is not None:
-                    M[i] = momentum * M[i] + g
-                    g = M[i]
-                mix = mix - lr * g
+            if o == NORMAL and not serial:
+                mix = mix - lr * direction(k, i)
             new[(i, k + 1)] = mix
         for (i, v), x in new.items():
             X[(i, v)] = x

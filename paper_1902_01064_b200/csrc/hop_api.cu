@@ -19,7 +19,9 @@ struct hop_ctx {
     int64_t P = 0;
     int32_t s = 0;
     // options
-    double lr = 0.1, momentum = 0.0, sigma = 1e-3;
+    double lr = 0.1, momentum = 0.0, sigma = 1e-3, weight_decay = 0.0;
+    int32_t loss = HOP_LOSS_HINGE;
+    bool serial = false;             // serial approach: Apply before Send (Section 3.2)
     int32_t grad_mode = HOP_GRAD_EXTERNAL, mix_kernel = HOP_MIX_AUTO;
     uint64_t grad_seed = 0;
     int64_t col_offset = 0;
@@ -43,7 +45,8 @@ struct hop_ctx {
     bool tc_maps_ready = false;
     // hop_run: instantiated CUDA graphs of level ranges, keyed by (first level, count)
     bool use_graph = true;
-    std::map<std::pair<int32_t, int32_t>, cudaGraphExec_t> graphs;
+    struct Graph { cudaGraphExec_t exec; int64_t launches; };
+    std::map<std::pair<int32_t, int32_t>, Graph> graphs;
     int32_t* d_i32 = nullptr;       // src_row and grad_workers of all levels
     HopRecord* d_rec = nullptr;
     HopEntry* d_ent = nullptr;
@@ -119,7 +122,7 @@ extern "C" int hop_create(hop_ctx** out, const int32_t* in_ptr, const int32_t* i
 
 // Kernel arguments (pointers, learning rate, tables) are baked into captured graphs: drop them on any change.
 static void drop_graphs(hop_ctx* c) {
-    for (auto& kv : c->graphs) cudaGraphExecDestroy(kv.second);
+    for (auto& kv : c->graphs) cudaGraphExecDestroy(kv.second.exec);
     c->graphs.clear();
 }
 
@@ -155,6 +158,21 @@ extern "C" int hop_set_option(hop_ctx* c, int key, double v) {
     drop_graphs(c);
     if (key == HOP_OPT_USE_GRAPH) { c->use_graph = v != 0.0; return HOP_OK; }
     if (key == HOP_OPT_NOTIFY_ACK) { c->sp.notify_ack = v != 0.0; return HOP_OK; }
+    if (key == HOP_OPT_WEIGHT_DECAY) {
+        if (v < 0) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: weight decay must be non-negative");
+        c->weight_decay = v;
+        return HOP_OK;
+    }
+    if (key == HOP_OPT_LOSS) {
+        if (v != HOP_LOSS_HINGE && v != HOP_LOSS_LOG) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: unknown loss");
+        c->loss = (int32_t)v;
+        return HOP_OK;
+    }
+    if (key == HOP_OPT_APPROACH) {
+        if (v != HOP_APPROACH_PARALLEL && v != HOP_APPROACH_SERIAL) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: unknown approach");
+        c->serial = v == HOP_APPROACH_SERIAL;
+        return HOP_OK;
+    }
     if (key == HOP_OPT_BACKUP_MODE) {
         if (v != HOP_BACKUP_AT_LEAST && v != HOP_BACKUP_EXACT) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: unknown backup mode");
         c->sp.backup_exact = (int32_t)v;
@@ -258,13 +276,16 @@ extern "C" int hop_bind_svm_csr(hop_ctx* c, const int64_t* row_ptr, const int32_
 
 // Tile width and kernel for one level: as many columns per tile as the staged rows leave room for.
 static int plan_level(hop_ctx* c, HopLevelHost& L, bool allow_tensor = true) {
-    const bool use_g = c->grad_mode != HOP_GRAD_SVM_CSR;
-    const bool mom = c->momentum != 0.0;
+    // In the serial approach gradient, momentum and weight decay are applied to x_k before the mix, which then only averages.
+    const bool use_g = c->grad_mode != HOP_GRAD_SVM_CSR && !c->serial;
+    const bool mom = c->momentum != 0.0 && !c->serial;
+    const bool decay = c->weight_decay != 0.0 && !c->serial;
     const int nG = use_g ? L.nG : 0;
     L.stage_rows = L.U + nG * (mom ? 2 : 1);
     int kernel = c->mix_kernel;
     // Tensor-core path: dense levels only (a contraction over <= 256 distinct slices for <= 128 workers).
-    const bool tc_ok = allow_tensor && c->g.N <= 128 && L.U <= 256 && L.nA > 0 && c->P % 128 == 0 && !mom && (use_g || L.nG == 0) &&
+    const bool tc_ok = allow_tensor && c->g.N <= 128 && L.U <= 256 && L.nA > 0 && c->P % 128 == 0 && !mom && !decay &&
+                       (use_g || L.nG == 0 || c->serial) &&
                        hop_dense_tc_smem((L.U + 31) / 32 * 32) > 0;
     const bool dense = L.nA >= 32 && L.sumC >= 32 * (int64_t)L.nA;
     if (tc_ok && (kernel == HOP_MIX_TENSOR || (kernel == HOP_MIX_AUTO && dense))) {
@@ -306,6 +327,7 @@ static int plan_level(hop_ctx* c, HopLevelHost& L, bool allow_tensor = true) {
     L.tile_w = (int32_t)w;
     L.kernel = kernel;
     for (HopEntry& e : L.ents) e.u *= L.tile_w;     // slice index -> float offset of its row in a staged tile
+    for (HopRecord& r : L.recs) if (r.self_u >= 0) r.self_u *= L.tile_w;
     // every distinct consumed slice once + gradient once + result once (+ momentum read and write)
     L.alg_bytes = 4 * c->P * ((int64_t)L.U + nG + L.nA + (mom ? 2 * (int64_t)nG : 0));
     return HOP_OK;
@@ -377,6 +399,8 @@ static int check_mode(hop_ctx* c) {
     if (mom && !c->M) HOP_FAIL(c, HOP_E_STATE, "momentum != 0 but no momentum buffer bound");
     if (c->grad_mode != HOP_GRAD_SVM_CSR && !c->G) HOP_FAIL(c, HOP_E_STATE, "this gradient mode needs a dense gradient buffer G");
     if (c->grad_mode == HOP_GRAD_SVM_CSR && mom) HOP_FAIL(c, HOP_E_UNSUPPORTED, "momentum with the CSR SVM mode is not implemented");
+    if (c->grad_mode == HOP_GRAD_SVM_CSR && c->serial && c->weight_decay != 0.0)
+        HOP_FAIL(c, HOP_E_UNSUPPORTED, "weight decay with the CSR SVM mode in the serial approach is not implemented");
     if (c->grad_mode == HOP_GRAD_SVM_CSR && !c->svmRowPtr) HOP_FAIL(c, HOP_E_STATE, "CSR SVM mode without hop_bind_svm_csr");
     if (c->grad_mode == HOP_GRAD_SVM_DENSE && !c->svmA) HOP_FAIL(c, HOP_E_STATE, "dense SVM mode without hop_bind_svm_dense");
     return HOP_OK;
@@ -413,7 +437,7 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, c
     size_t t0 = 0, t1 = 0;
     HopLaunchCfg cfg{};
     cfg.X = c->X; cfg.M = c->M; cfg.G = c->G; cfg.P = c->P; cfg.N = c->g.N; cfg.s = c->s;
-    cfg.lr = (float)c->lr; cfg.mu = (float)c->momentum; cfg.tile_w = L.tile_w;
+    cfg.lr = (float)c->lr; cfg.mu = (float)c->momentum; cfg.wd = (float)c->weight_decay; cfg.loss = c->loss; cfg.tile_w = L.tile_w;
     cfg.use_g = c->grad_mode != HOP_GRAD_SVM_CSR;
     cfg.sm_count = c->sm_count; cfg.err_word = c->d_err; cfg.stream = c->stream;
     cfg.table_smem = L.table_smem; cfg.n_ents = (int32_t)L.ents.size();
@@ -432,6 +456,17 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, c
         if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("gradient kernel launch: ") + cudaGetErrorString((cudaError_t)e));
         HOP_SPAN_END(0, 0);
     }
+    if (c->serial && L.nG > 0) {      // Apply on x_k before it is sent: dense update kernel, or the sparse apply on slot k
+        HOP_SPAN_BEGIN();
+        if (c->grad_mode == HOP_GRAD_SVM_CSR)
+            e = hop_launch_svm_csr_apply(cfg, lv, c->svmRowPtr, c->svmCol, c->svmVal, c->svmR, c->svmB, c->coef, 0);
+        else
+            e = hop_launch_apply_dense(cfg, lv);
+        c->launches += 1;
+        if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("apply launch: ") + cudaGetErrorString((cudaError_t)e));
+        HOP_SPAN_END(2, 0);
+        cfg.use_g = 0; cfg.mu = 0.f; cfg.wd = 0.f;      // the mix only averages
+    }
     if (L.nA > 0) {
         HOP_SPAN_BEGIN();
         if (L.kernel == HOP_MIX_TENSOR)
@@ -444,9 +479,9 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, c
         if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("mix kernel launch: ") + cudaGetErrorString((cudaError_t)e));
         HOP_SPAN_END(1, L.alg_bytes);
     }
-    if (L.nG > 0 && c->grad_mode == HOP_GRAD_SVM_CSR) {
+    if (L.nG > 0 && c->grad_mode == HOP_GRAD_SVM_CSR && !c->serial) {
         HOP_SPAN_BEGIN();
-        e = hop_launch_svm_csr_apply(cfg, lv, c->svmRowPtr, c->svmCol, c->svmVal, c->svmR, c->svmB, c->coef);
+        e = hop_launch_svm_csr_apply(cfg, lv, c->svmRowPtr, c->svmCol, c->svmVal, c->svmR, c->svmB, c->coef, 1);
         c->launches += 1;
         if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("sparse apply launch: ") + cudaGetErrorString((cudaError_t)e));
         HOP_SPAN_END(2, 0);
@@ -499,6 +534,7 @@ extern "C" int hop_run(hop_ctx* c, int32_t n_levels) {
             for (int32_t k = first; k < first + n_levels && !rc; ++k) rc = enqueue_level(c, k);
             cudaGraph_t g = nullptr;
             const cudaError_t ce = cudaStreamEndCapture(c->stream, &g);
+            const int64_t in_graph = c->launches - launches_before;
             c->launches = launches_before;
             if (rc) { if (g) cudaGraphDestroy(g); return rc; }
             if (ce != cudaSuccess) { c->err = std::string("hop_run: stream capture: ") + cudaGetErrorString(ce); return HOP_E_CUDA; }
@@ -506,13 +542,10 @@ extern "C" int hop_run(hop_ctx* c, int32_t n_levels) {
             const cudaError_t ie = cudaGraphInstantiate(&ex, g, 0);
             cudaGraphDestroy(g);
             if (ie != cudaSuccess) { c->err = std::string("hop_run: graph instantiation: ") + cudaGetErrorString(ie); return HOP_E_CUDA; }
-            it = c->graphs.emplace(key, ex).first;
+            it = c->graphs.emplace(key, hop_ctx::Graph{ex, in_graph}).first;
         }
-        HOP_CUDA(c, cudaGraphLaunch(it->second, c->stream));
-        for (int32_t k = first; k < first + n_levels; ++k) {
-            const HopLevelHost& L = c->levels[k];
-            c->launches += (L.nA > 0) + (L.nG > 0 ? (c->grad_mode == HOP_GRAD_SVM_DENSE ? 2 : c->grad_mode == HOP_GRAD_SVM_CSR ? 2 : 1) : 0);
-        }
+        HOP_CUDA(c, cudaGraphLaunch(it->second.exec, c->stream));
+        c->launches += it->second.launches;
     }
     for (int32_t k = first; k < first + n_levels; ++k)
         for (const HopRecord& r : c->levels[k].recs) c->newest[r.worker] = k + 1;

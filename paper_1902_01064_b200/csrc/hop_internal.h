@@ -23,7 +23,8 @@ struct HopRecord {          // one active (NORMAL or JUMP) worker of a level
     int32_t ent_count;
     int32_t g_stage;        // index among the level's NORMAL workers, -1 for JUMP
     int32_t cur_row;        // row of X holding x_{k,i} (gradient input); -1 for JUMP
-    int32_t pad0, pad1;
+    int32_t self_u;         // float offset of the worker's own consumed slice inside a staged tile (weight decay)
+    int32_t pad1;
 };
 struct HopEntry {
     int32_t u;              // float offset of the slice's row inside a staged tile: slice index * tile width
@@ -115,6 +116,8 @@ struct HopLaunchCfg {
     int64_t P;
     int32_t N, s;
     float lr, mu;
+    float wd;           // weight decay lambda: lambda * x_{k,i} joins the gradient of NORMAL records
+    int32_t loss;       // 0 hinge, 1 log (SVM modes)
     int32_t tile_w;
     int32_t use_g;      // dense gradient rows are applied
     int32_t sm_count;
@@ -130,8 +133,11 @@ int hop_launch_svm_dense(const HopLaunchCfg& c, const HopLevelDev& lv, const flo
                          int32_t R, int32_t B, float* coef);
 int hop_launch_svm_csr_coef(const HopLaunchCfg& c, const HopLevelDev& lv, const int64_t* row_ptr, const int32_t* col,
                             const float* val, const float* y, int32_t R, int32_t B, float* coef);
+// slot_shift 1: apply to x_{k+1} after the mix (parallel approach); 0: to x_k before it (serial approach)
 int hop_launch_svm_csr_apply(const HopLaunchCfg& c, const HopLevelDev& lv, const int64_t* row_ptr, const int32_t* col,
-                             const float* val, int32_t R, int32_t B, const float* coef);
+                             const float* val, int32_t R, int32_t B, const float* coef, int32_t slot_shift);
+// serial approach, dense gradients: x_k <- x_k - lr * d in place for the level's NORMAL workers
+int hop_launch_apply_dense(const HopLaunchCfg& c, const HopLevelDev& lv);
 int hop_mix_smem_budget(int kernel);   // usable dynamic shared memory per CTA for the kernel
 int hop_mix_stages(int kernel);
 int hop_mix_table_limit();

@@ -29,15 +29,18 @@ enum : int32_t { ERR_FULL_WAIT = 1 << 24, ERR_EMPTY_WAIT = 2 << 24 };
 // ------------------------------------------------------------------------------------------------
 // Consumer math shared by both mix kernels: one warp produces the tile of one record.
 // stage: [rows][w] floats; rows [0,U) consumed slices, [U,U+nG) gradients, [U+nG,U+2nG) momentum.
-template <int VEC, bool MOMENTUM>
+template <int VEC, bool MOMENTUM, bool DECAY>
 __device__ __forceinline__ void reduce_apply_record(const HopRecord& r, const HopEntry* __restrict__ ents,
                                                     const float* __restrict__ stage, int w, int wd, int U, int nG,
-                                                    bool use_g, float lr, float mu, float* __restrict__ X,
+                                                    bool use_g, float lr, float mu, float lam, float* __restrict__ X,
                                                     float* __restrict__ M, int64_t P, int64_t c0, int lane) {
     const HopEntry* e = ents + r.ent_begin;
     const int n = r.ent_count;
     float* out = X + (int64_t)r.out_row * P + c0;
     const bool grad = use_g && r.g_stage >= 0;
+    // weight decay: lambda * x_{k,i} joins the gradient; x_{k,i} is the worker's own consumed slice.  With a sparse
+    // gradient (no dense row) only the decay term is applied here, the data term by the sparse apply.
+    const bool decay = DECAY && r.g_stage >= 0 && r.self_u >= 0;   // DECAY is a template flag: the common path carries no trace of it
     const float* grow = stage + (int64_t)(U + (grad ? r.g_stage : 0)) * w;
     const float* mrow = stage + (int64_t)(U + nG + (grad ? r.g_stage : 0)) * w;
     float* mout = MOMENTUM ? (M + (int64_t)r.worker * P + c0) : nullptr;
@@ -61,8 +64,17 @@ __device__ __forceinline__ void reduce_apply_record(const HopRecord& r, const Ho
                 HOP_FMA4(en.w, v);
             }
 #undef HOP_FMA4
+            if (decay && !grad) {
+                const float4 xs = *reinterpret_cast<const float4*>(sc + r.self_u);
+                const float k = -lr * lam;
+                acc.x = fmaf(k, xs.x, acc.x); acc.y = fmaf(k, xs.y, acc.y); acc.z = fmaf(k, xs.z, acc.z); acc.w = fmaf(k, xs.w, acc.w);
+            }
             if (grad) {
                 float4 g = *reinterpret_cast<const float4*>(grow + c);
+                if (decay) {
+                    const float4 xs = *reinterpret_cast<const float4*>(sc + r.self_u);
+                    g.x = fmaf(lam, xs.x, g.x); g.y = fmaf(lam, xs.y, g.y); g.z = fmaf(lam, xs.z, g.z); g.w = fmaf(lam, xs.w, g.w);
+                }
                 if constexpr (MOMENTUM) {
                     const float4 m = *reinterpret_cast<const float4*>(mrow + c);
                     g.x = fmaf(mu, m.x, g.x); g.y = fmaf(mu, m.y, g.y);
@@ -79,8 +91,10 @@ __device__ __forceinline__ void reduce_apply_record(const HopRecord& r, const Ho
                 const HopEntry en = e[t];
                 acc = fmaf(en.w, stage[en.u + c], acc);
             }
+            if (decay && !grad) acc = fmaf(-lr * lam, stage[r.self_u + c], acc);
             if (grad) {
                 float g = grow[c];
+                if (decay) g = fmaf(lam, stage[r.self_u + c], g);
                 if constexpr (MOMENTUM) {
                     g = fmaf(mu, mrow[c], g);
                     mout[c] = g;
@@ -95,10 +109,10 @@ __device__ __forceinline__ void reduce_apply_record(const HopRecord& r, const Ho
 // ------------------------------------------------------------------------------------------------
 // mix_staged: ordinary loads into shared memory, one barrier, compute, one barrier.  Works for any P
 // (VEC = 1 when P is not a multiple of 4).
-template <int VEC, bool MOMENTUM>
+template <int VEC, bool MOMENTUM, bool DECAY>
 __global__ void __launch_bounds__(kStagedThreads)
 mix_staged_kernel(float* __restrict__ X, float* __restrict__ M, const float* __restrict__ G, int64_t P, int w,
-                  int use_g, float lr, float mu, HopLevelDev lv) {
+                  int use_g, float lr, float mu, float lam, HopLevelDev lv) {
     extern __shared__ __align__(16) float smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nG = use_g ? lv.nG : 0;
@@ -121,7 +135,7 @@ mix_staged_kernel(float* __restrict__ X, float* __restrict__ M, const float* __r
         }
         __syncthreads();
         for (int a = warp; a < lv.nA; a += kStagedThreads / 32)
-            reduce_apply_record<VEC, MOMENTUM>(lv.recs[a], lv.ents, smem, w, wd, lv.U, nG, use_g != 0, lr, mu, X, M, P, c0, lane);
+            reduce_apply_record<VEC, MOMENTUM, DECAY>(lv.recs[a], lv.ents, smem, w, wd, lv.U, nG, use_g != 0, lr, mu, lam, X, M, P, c0, lane);
         __syncthreads();
     }
 }
@@ -161,10 +175,10 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 // every staged row of the next tile, rows dealt round-robin to the producer lanes, completion counted
 // in bytes on an mbarrier), the other kConsumerWarps warps consume.  Two stages.
 // Requires P % 4 == 0 and 16-byte aligned base pointers (bulk copies move multiples of 16 bytes).
-template <bool MOMENTUM>
+template <bool MOMENTUM, bool DECAY>
 __global__ void __launch_bounds__(kBulkThreads, 1)
 mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __restrict__ G, int64_t P, int w,
-                int use_g, float lr, float mu, HopLevelDev lv, int table_bytes, int n_ents,
+                int use_g, float lr, float mu, float lam, HopLevelDev lv, int table_bytes, int n_ents,
                 int32_t* __restrict__ err_word) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw);
@@ -234,7 +248,7 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
             const int wd = (int)min((int64_t)w, P - c0);
             const float* st = stage0 + s * stage_floats;
             for (int a = cw; a < lv.nA; a += kConsumerWarps)
-                reduce_apply_record<4, MOMENTUM>(recs[a], ents, st, w, wd, lv.U, nG, use_g != 0, lr, mu, X, M, P, c0, lane);
+                reduce_apply_record<4, MOMENTUM, DECAY>(recs[a], ents, st, w, wd, lv.U, nG, use_g != 0, lr, mu, lam, X, M, P, c0, lane);
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[s]);
         }
@@ -304,10 +318,16 @@ __device__ __forceinline__ double warp_sum(double v) {
     return v;
 }
 
+// d(loss)/d(margin) of one row: hinge -y/B on the active set (y*m < 1, strict), log loss -y / (B (1 + e^{y m})).
+__device__ __forceinline__ float loss_coefficient(float y, double m, int B, int loss) {
+    if (loss == 0) return ((double)y * m < 1.0) ? -y / (float)B : 0.f;
+    return (float)(-(double)y / ((double)B * (1.0 + exp((double)y * m))));
+}
+
 __global__ void __launch_bounds__(256)
 svm_margin_csr_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelDev lv, const int64_t* __restrict__ row_ptr,
                       const int32_t* __restrict__ col, const float* __restrict__ val, const float* __restrict__ y,
-                      int R, int B, float* __restrict__ coef) {
+                      int R, int B, int loss, float* __restrict__ coef) {
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (gw >= lv.nG * B) return;
     const int a = gw / B, r = gw - a * B;
@@ -317,15 +337,12 @@ svm_margin_csr_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelDev
     double m = 0.0;
     for (int64_t t = row_ptr[row] + lane; t < row_ptr[row + 1]; t += 32) m += (double)val[t] * (double)x[col[t]];
     m = warp_sum(m);
-    if (lane == 0) {
-        const float yy = y[(int64_t)worker * R + (row - (int64_t)worker * R)];
-        coef[(int64_t)worker * B + r] = ((double)yy * m < 1.0) ? -yy / (float)B : 0.f;
-    }
+    if (lane == 0) coef[(int64_t)worker * B + r] = loss_coefficient(y[row], m, B, loss);
 }
 
 __global__ void __launch_bounds__(256)
 svm_margin_dense_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelDev lv, const float* __restrict__ A,
-                        const float* __restrict__ y, int R, int B, float* __restrict__ coef) {
+                        const float* __restrict__ y, int R, int B, int loss, float* __restrict__ coef) {
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (gw >= lv.nG * B) return;
     const int a = gw / B, r = gw - a * B;
@@ -336,10 +353,7 @@ svm_margin_dense_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelD
     double m = 0.0;
     for (int64_t p = lane; p < P; p += 32) m += (double)arow[p] * (double)x[p];
     m = warp_sum(m);
-    if (lane == 0) {
-        const float yy = y[row];
-        coef[(int64_t)worker * B + r] = ((double)yy * m < 1.0) ? -yy / (float)B : 0.f;
-    }
+    if (lane == 0) coef[(int64_t)worker * B + r] = loss_coefficient(y[row], m, B, loss);
 }
 
 // g[i][p] = sum_r coef_r * A[r][p]; one thread per column, rows of the minibatch in order.
@@ -360,7 +374,7 @@ svm_dense_grad_kernel(float* __restrict__ G, int64_t P, HopLevelDev lv, const fl
 __global__ void __launch_bounds__(256)
 svm_csr_apply_kernel(float* __restrict__ X, int64_t P, int S, float lr, HopLevelDev lv, const int64_t* __restrict__ row_ptr,
                      const int32_t* __restrict__ col, const float* __restrict__ val, int R, int B,
-                     const float* __restrict__ coef) {
+                     const float* __restrict__ coef, int slot_shift) {
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (gw >= lv.nG * B) return;
     const int a = gw / B, r = gw - a * B;
@@ -368,9 +382,41 @@ svm_csr_apply_kernel(float* __restrict__ X, int64_t P, int S, float lr, HopLevel
     const float cf = coef[(int64_t)worker * B + r];
     if (cf == 0.f) return;
     const int64_t row = (int64_t)worker * R + (int64_t)(lv.level % (R / B)) * B + r;
-    float* x = X + ((int64_t)worker * S + (lv.level + 1) % S) * P;
+    float* x = X + ((int64_t)worker * S + (lv.level + slot_shift) % S) * P;
     const float scale = -lr * cf;
     for (int64_t t = row_ptr[row] + lane; t < row_ptr[row + 1]; t += 32) atomicAdd(x + col[t], scale * val[t]);
+}
+
+// Serial approach (Compute, Apply, then Send): x_k <- x_k - lr * d in place for the level's NORMAL workers, with
+// d = g (+ lambda x_k), through the momentum buffer when there is one.  One float4 per thread.
+template <bool MOMENTUM>
+__global__ void __launch_bounds__(256)
+apply_dense_kernel(float* __restrict__ X, float* __restrict__ M, const float* __restrict__ G, int64_t P, int S, float lr,
+                   float mu, float lam, HopLevelDev lv) {
+    const int worker = lv.grad_workers[blockIdx.y];
+    const int64_t c = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (c >= P) return;
+    float* x = X + ((int64_t)worker * S + lv.level % S) * P + c;
+    const float* g = G + (int64_t)worker * P + c;
+    float* m = MOMENTUM ? M + (int64_t)worker * P + c : nullptr;
+    const int n = (int)min((int64_t)4, P - c);
+    if (n == 4 && (P & 3) == 0) {
+        float4 xv = *reinterpret_cast<float4*>(x), gv = *reinterpret_cast<const float4*>(g);
+        gv.x = fmaf(lam, xv.x, gv.x); gv.y = fmaf(lam, xv.y, gv.y); gv.z = fmaf(lam, xv.z, gv.z); gv.w = fmaf(lam, xv.w, gv.w);
+        if constexpr (MOMENTUM) {
+            const float4 mv = *reinterpret_cast<float4*>(m);
+            gv.x = fmaf(mu, mv.x, gv.x); gv.y = fmaf(mu, mv.y, gv.y); gv.z = fmaf(mu, mv.z, gv.z); gv.w = fmaf(mu, mv.w, gv.w);
+            *reinterpret_cast<float4*>(m) = gv;
+        }
+        xv.x = fmaf(-lr, gv.x, xv.x); xv.y = fmaf(-lr, gv.y, xv.y); xv.z = fmaf(-lr, gv.z, xv.z); xv.w = fmaf(-lr, gv.w, xv.w);
+        *reinterpret_cast<float4*>(x) = xv;
+    } else {
+        for (int e = 0; e < n; ++e) {
+            float gv = fmaf(lam, x[e], g[e]);
+            if constexpr (MOMENTUM) { gv = fmaf(mu, m[e], gv); m[e] = gv; }
+            x[e] = fmaf(-lr, gv, x[e]);
+        }
+    }
 }
 
 size_t staged_smem(const HopLaunchCfg& c, const HopLevelDev& lv) {
@@ -395,16 +441,18 @@ int hop_launch_mix_staged(const HopLaunchCfg& c, const HopLevelDev& lv) {
     const bool mom = c.mu != 0.f;
     cudaStream_t st = (cudaStream_t)c.stream;
     cudaError_t e = cudaSuccess;
-#define HOP_LAUNCH_STAGED(V, MO)                                                                              \
+#define HOP_LAUNCH_STAGED(V, MO, DE)                                                                          \
     do {                                                                                                      \
-        e = hop_allow_max_smem<mix_staged_kernel<V, MO>>();                                                   \
+        e = hop_allow_max_smem<mix_staged_kernel<V, MO, DE>>();                                               \
         if (e == cudaSuccess)                                                                                 \
-            mix_staged_kernel<V, MO><<<grid, kStagedThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, lv); \
+            mix_staged_kernel<V, MO, DE><<<grid, kStagedThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, c.wd, lv); \
     } while (0)
-    if (vec && mom) HOP_LAUNCH_STAGED(4, true);
-    else if (vec) HOP_LAUNCH_STAGED(4, false);
-    else if (mom) HOP_LAUNCH_STAGED(1, true);
-    else HOP_LAUNCH_STAGED(1, false);
+#define HOP_LAUNCH_STAGED2(V, MO) do { if (c.wd != 0.f) HOP_LAUNCH_STAGED(V, MO, true); else HOP_LAUNCH_STAGED(V, MO, false); } while (0)
+    if (vec && mom) HOP_LAUNCH_STAGED2(4, true);
+    else if (vec) HOP_LAUNCH_STAGED2(4, false);
+    else if (mom) HOP_LAUNCH_STAGED2(1, true);
+    else HOP_LAUNCH_STAGED2(1, false);
+#undef HOP_LAUNCH_STAGED2
 #undef HOP_LAUNCH_STAGED
     if (e != cudaSuccess) return (int)e;
     return (int)cudaGetLastError();
@@ -418,16 +466,21 @@ int hop_launch_mix_bulk(const HopLaunchCfg& c, const HopLevelDev& lv) {
     const int64_t tiles = (c.P + c.tile_w - 1) / c.tile_w;
     const int grid = (int)std::min<int64_t>(tiles, (int64_t)c.sm_count);
     cudaStream_t st = (cudaStream_t)c.stream;
-    cudaError_t e;
-    if (c.mu != 0.f) {
-        e = hop_allow_max_smem<mix_bulk_kernel<true>>();
-        if (e != cudaSuccess) return (int)e;
-        mix_bulk_kernel<true><<<grid, kBulkThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, lv, c.table_smem, c.n_ents, c.err_word);
-    } else {
-        e = hop_allow_max_smem<mix_bulk_kernel<false>>();
-        if (e != cudaSuccess) return (int)e;
-        mix_bulk_kernel<false><<<grid, kBulkThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, lv, c.table_smem, c.n_ents, c.err_word);
-    }
+    cudaError_t e = cudaSuccess;
+#define HOP_LAUNCH_BULK(MO, DE)                                                                               \
+    do {                                                                                                      \
+        e = hop_allow_max_smem<mix_bulk_kernel<MO, DE>>();                                                    \
+        if (e == cudaSuccess)                                                                                 \
+            mix_bulk_kernel<MO, DE><<<grid, kBulkThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, c.wd, lv, \
+                                                                      c.table_smem, c.n_ents, c.err_word);   \
+    } while (0)
+    const bool mom = c.mu != 0.f, dec = c.wd != 0.f;
+    if (mom && dec) HOP_LAUNCH_BULK(true, true);
+    else if (mom) HOP_LAUNCH_BULK(true, false);
+    else if (dec) HOP_LAUNCH_BULK(false, true);
+    else HOP_LAUNCH_BULK(false, false);
+#undef HOP_LAUNCH_BULK
+    if (e != cudaSuccess) return (int)e;
     return (int)cudaGetLastError();
 }
 
@@ -443,7 +496,7 @@ int hop_launch_svm_dense(const HopLaunchCfg& c, const HopLevelDev& lv, const flo
                          int32_t R, int32_t B, float* coef) {
     if (lv.nG == 0) return 0;
     const int warps = lv.nG * B;
-    svm_margin_dense_kernel<<<(warps * 32 + 255) / 256, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.P, c.s + 1, lv, A, y, R, B, coef);
+    svm_margin_dense_kernel<<<(warps * 32 + 255) / 256, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.P, c.s + 1, lv, A, y, R, B, c.loss, coef);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return (int)e;
     dim3 grid((unsigned)((c.P + 255) / 256), (unsigned)lv.nG);
@@ -455,14 +508,22 @@ int hop_launch_svm_csr_coef(const HopLaunchCfg& c, const HopLevelDev& lv, const 
                             const float* val, const float* y, int32_t R, int32_t B, float* coef) {
     if (lv.nG == 0) return 0;
     const int warps = lv.nG * B;
-    svm_margin_csr_kernel<<<(warps * 32 + 255) / 256, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.P, c.s + 1, lv, row_ptr, col, val, y, R, B, coef);
+    svm_margin_csr_kernel<<<(warps * 32 + 255) / 256, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.P, c.s + 1, lv, row_ptr, col, val, y, R, B, c.loss, coef);
     return (int)cudaGetLastError();
 }
 
 int hop_launch_svm_csr_apply(const HopLaunchCfg& c, const HopLevelDev& lv, const int64_t* row_ptr, const int32_t* col,
-                             const float* val, int32_t R, int32_t B, const float* coef) {
+                             const float* val, int32_t R, int32_t B, const float* coef, int32_t slot_shift) {
     if (lv.nG == 0) return 0;
     const int warps = lv.nG * B;
-    svm_csr_apply_kernel<<<(warps * 32 + 255) / 256, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.P, c.s + 1, c.lr, lv, row_ptr, col, val, R, B, coef);
+    svm_csr_apply_kernel<<<(warps * 32 + 255) / 256, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.P, c.s + 1, c.lr, lv, row_ptr, col, val, R, B, coef, slot_shift);
+    return (int)cudaGetLastError();
+}
+
+int hop_launch_apply_dense(const HopLaunchCfg& c, const HopLevelDev& lv) {
+    if (lv.nG == 0) return 0;
+    dim3 grid((unsigned)(((c.P + 3) / 4 + 255) / 256), (unsigned)lv.nG);
+    if (c.mu != 0.f) apply_dense_kernel<true><<<grid, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.M, c.G, c.P, c.s + 1, c.lr, c.mu, c.wd, lv);
+    else apply_dense_kernel<false><<<grid, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.M, c.G, c.P, c.s + 1, c.lr, c.mu, c.wd, lv);
     return (int)cudaGetLastError();
 }

@@ -129,9 +129,11 @@ void hop_build_level(const HopGraph& g, int32_t s, int32_t level, const int32_t*
             r.cur_row = -1;
             ++out.nJump;
         }
+        r.self_u = -1;
         for (int64_t t = ptr[i]; t < ptr[i + 1]; ++t) {
             const int32_t row = nbr[t] * S + ver[t] % S;
             if (slice_of[row] < 0) { slice_of[row] = out.U++; out.src_row.push_back(row); }
+            if (nbr[t] == i) r.self_u = slice_of[row];      // slice index for now; scaled by the tile width when planned
             out.ents.push_back({slice_of[row], (float)num[t] / (float)den[i]});
             out.ent_slice.push_back(slice_of[row]);
             out.ent_num.push_back(num[t]);

@@ -21,7 +21,10 @@ W_UNIFORM, W_STALE_LINEAR = 0, 1
 GRAD_EXTERNAL, GRAD_SYNTHETIC, GRAD_SVM_DENSE, GRAD_SVM_CSR = 0, 1, 2, 3
 MIX_AUTO, MIX_STAGED, MIX_BULK, MIX_TENSOR = 0, 1, 2, 3
 (OPT_MAX_IG, OPT_LR, OPT_MOMENTUM, OPT_WEIGHT_MODE, OPT_GRAD_MODE, OPT_GRAD_SEED, OPT_GRAD_SIGMA,
- OPT_MIX_KERNEL, OPT_COL_OFFSET, OPT_USE_GRAPH, OPT_BACKUP_MODE, OPT_NOTIFY_ACK) = range(1, 13)
+ OPT_MIX_KERNEL, OPT_COL_OFFSET, OPT_USE_GRAPH, OPT_BACKUP_MODE, OPT_NOTIFY_ACK, OPT_WEIGHT_DECAY, OPT_LOSS,
+ OPT_APPROACH) = range(1, 16)
+LOSS_HINGE, LOSS_LOG = 0, 1
+APPROACH_PARALLEL, APPROACH_SERIAL = 0, 1
 BACKUP_AT_LEAST, BACKUP_EXACT = 0, 1
 OPT_BACKUP_OF_WORKER = 1000
 

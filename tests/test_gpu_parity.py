@@ -18,8 +18,9 @@ KEYS = ("op", "ptr", "nbr", "ver", "num", "den")
 class GpuRun:
     """Device buffers (torch, plumbing only) + a configured context for a workload."""
 
-    def __init__(self, w, mix_kernel=hop.MIX_AUTO, x0=None, external_G=None):
+    def __init__(self, w, mix_kernel=hop.MIX_AUTO, x0=None, external_G=None, variant=None):
         self.w = w
+        self.variant = variant or {}
         S = w.s + 1
         self.X = torch.zeros((w.N, S, w.P), dtype=torch.float32, device=DEV)
         self.M = torch.zeros((w.N, w.P), dtype=torch.float32, device=DEV) if w.momentum else None
@@ -27,6 +28,9 @@ class GpuRun:
         self.h = hop.from_workload(w, mix_kernel)
         if external_G is not None:
             self.h.set_option(hop.OPT_GRAD_MODE, hop.GRAD_EXTERNAL)
+        self.h.set_option(hop.OPT_LOSS, hop.LOSS_LOG if self.variant.get("loss") == "log" else hop.LOSS_HINGE)
+        self.h.set_option(hop.OPT_WEIGHT_DECAY, self.variant.get("weight_decay", 0.0))
+        self.h.set_option(hop.OPT_APPROACH, hop.APPROACH_SERIAL if self.variant.get("serial") else hop.APPROACH_PARALLEL)
         self.external_G = external_G
         self.h.bind_buffers(self.X, self.M, self.G, torch.cuda.current_stream().cuda_stream)
         if w.grad_mode == inputs.GRAD_SVM_DENSE:
@@ -54,30 +58,33 @@ class GpuRun:
         return [self.h.read_params(i) for i in range(self.w.N)]
 
 
-def oracle_grad_fn(w, cols=None, external_G=None):
+def oracle_grad_fn(w, cols=None, external_G=None, loss="hinge"):
     if external_G is not None:
         return up.GradExternal(external_G if cols is None else external_G[:, :, cols])
     if w.grad_mode == inputs.GRAD_SYNTHETIC:
         return up.GradSynthetic(w.grad_seed, w.sigma, np.arange(w.P) if cols is None else cols)
     if w.grad_mode == inputs.GRAD_SVM_DENSE:
-        return up.GradSvmDense(w.svm.dense, w.svm.y, w.svm.batch)
-    return up.GradSvmCsr(w.svm.row_ptr, w.svm.col, w.svm.val, w.svm.y, w.svm.rows_per_worker, w.svm.batch)
+        return up.GradSvmDense(w.svm.dense, w.svm.y, w.svm.batch, loss)
+    return up.GradSvmCsr(w.svm.row_ptr, w.svm.col, w.svm.val, w.svm.y, w.svm.rows_per_worker, w.svm.batch, loss)
 
 
-def oracle_run(w, x0, levels, cols=None, external_G=None):
+def oracle_run(w, x0, levels, cols=None, external_G=None, variant=None):
+    variant = variant or {}
     tr = op.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode).to_arrays()
     xs = x0.astype(np.float64) if cols is None else x0[:, cols].astype(np.float64)
-    X, newest = up.run_updates(tr, w.N, w.lr, w.momentum, xs, oracle_grad_fn(w, cols, external_G), levels=levels, s=w.s)
+    X, newest = up.run_updates(tr, w.N, w.lr, w.momentum, xs, oracle_grad_fn(w, cols, external_G, variant.get("loss", "hinge")),
+                               levels=levels, s=w.s, weight_decay=variant.get("weight_decay", 0.0),
+                               serial=bool(variant.get("serial")))
     return tr, [X[(i, newest[i])] for i in range(w.N)], newest
 
 
-def check(w, levels, tol, mix_kernel=hop.MIX_AUTO, perturb=False, cols=None, external_G=None):
+def check(w, levels, tol, mix_kernel=hop.MIX_AUTO, perturb=False, cols=None, external_G=None, variant=None):
     x0 = np.tile(w.p0(), (w.N, 1))
     if perturb:
         x0 = np.stack([w.p0() + w.perturbation(i) for i in range(w.N)])
-    g = GpuRun(w, mix_kernel, x0, external_G)
+    g = GpuRun(w, mix_kernel, x0, external_G, variant)
     got = g.run(levels)
-    tr, want, newest = oracle_run(w, x0, levels, cols, external_G)
+    tr, want, newest = oracle_run(w, x0, levels, cols, external_G, variant)
     gt = g.trace.to_arrays()
     for k in KEYS:
         assert np.array_equal(gt[k], tr[k]), k                                  # traces bit-exact
@@ -366,4 +373,51 @@ def test_graph_replay_of_level_ranges_equals_step_by_step(cfg, P, iters):
         else:
             scale = np.abs(ref[i]).max() + 1e-30
             assert np.abs(first[i] - ref[i]).max() <= 1e-5 * scale and np.abs(second[i] - ref[i]).max() <= 1e-5 * scale
+    g.h.close()
+
+
+# ------------------------------------------------------------------ loss / regulariser / operation order variants
+VARIANTS = [dict(loss="log"), dict(weight_decay=0.05), dict(loss="log", weight_decay=0.02, serial=True), dict(serial=True)]
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_dense_svm_with_log_loss_weight_decay_momentum_and_serial_order(kernel, variant):
+    # the paper's SVM runs: log loss, momentum 0.9, weight decay (Section 7.2)
+    w = inputs.make_workload(1)
+    w.momentum = 0.9
+    check(w, w.iters, TOL_RUN, kernel, variant=variant)
+    check(w, 1, TOL_STEP, kernel, perturb=True, variant=variant)
+
+
+@pytest.mark.parametrize("variant", [dict(loss="log"), dict(weight_decay=0.05), dict(loss="log", serial=True)])
+def test_csr_svm_variants(variant):
+    w = inputs.make_workload(2, P=8192, iters=60)
+    check(w, w.iters, TOL_RUN, variant=variant)
+    check(w, 1, TOL_STEP, perturb=True, variant=variant)
+
+
+@pytest.mark.parametrize("variant", [dict(serial=True), dict(weight_decay=0.01), dict(serial=True, weight_decay=0.01)])
+def test_synthetic_gradient_variants_with_momentum_and_jumps(variant):
+    w = inputs.make_workload(3, P=5000, iters=60)
+    for kernel in KERNELS:
+        check(w, w.iters, TOL_RUN, kernel, variant=variant)
+        check(w, 1, TOL_STEP, kernel, perturb=True, variant=variant)
+
+
+def test_tensor_path_in_serial_order():
+    w = inputs.make_workload(5, P=1536, iters=10)
+    g = GpuRun(w, hop.MIX_TENSOR, variant=dict(serial=True))
+    assert g.h.level_stats(2)["kernel"] == hop.MIX_TENSOR
+    g.h.close()
+    check(w, w.iters, TOL_RUN, hop.MIX_TENSOR, variant=dict(serial=True))
+    check(w, 1, TOL_STEP, hop.MIX_TENSOR, perturb=True, variant=dict(serial=True))
+
+
+def test_unsupported_combinations_are_refused():
+    w = inputs.make_workload(2, P=4096, iters=4)
+    g = GpuRun(w, variant=dict(serial=True, weight_decay=0.1))
+    with pytest.raises(hop.HopError) as e:
+        g.h.step()
+    assert e.value.code == hop.E_UNSUPPORTED
     g.h.close()

@@ -225,3 +225,63 @@ def test_synthetic_gradient_is_a_pure_function_of_its_indices():
     assert not np.allclose(g, philox.synthetic_gradient(12345678901, 3, 8, cols, 1e-3))
     big = philox.synthetic_gradient(99, 0, 0, np.arange(400000), 1e-3)
     assert abs(big.mean()) < 1e-5 and abs(big.std() - 1e-3) < 1e-5
+
+
+# ------------------------------------------------------------------ log loss, weight decay, serial approach
+def test_log_loss_gradient_matches_autograd_and_finite_differences():
+    rng = np.random.default_rng(11)
+    A = rng.standard_normal((32, 10)).astype(np.float32)
+    y = np.where(rng.random(32) < 0.5, -1.0, 1.0).astype(np.float32)
+    x = rng.standard_normal(10)
+    g = up.svm_gradient_dense(A, y, x, loss="log")
+    xt = torch.tensor(x, dtype=torch.float64, requires_grad=True)
+    loss = torch.nn.functional.softplus(-torch.tensor(y, dtype=torch.float64) * (torch.tensor(A, dtype=torch.float64) @ xt)).mean()
+    loss.backward()
+    np.testing.assert_allclose(g, xt.grad.numpy(), atol=1e-13)
+    h = 1e-6
+    for p in range(10):
+        e = np.zeros(10)
+        e[p] = h
+        fd = (up.mean_log_loss(A, y, x + e) - up.mean_log_loss(A, y, x - e)) / (2 * h)
+        assert abs(fd - g[p]) < 1e-8
+
+
+def test_weight_decay_and_momentum_match_torch_sgd_single_worker():
+    rng = np.random.default_rng(12)
+    C, iters, lr, mu, wd = 9, 10, 0.1, 0.9, 0.05
+    x0 = rng.standard_normal((1, C))
+    G = rng.standard_normal((iters, 1, C))
+    tr = trace_equal_speed([[0]], iters)
+    for serial in (False, True):                        # with one worker Reduce is the identity: both orders coincide
+        X, _ = up.run_updates(tr, 1, lr, mu, x0, up.GradExternal(G), keep_all=True, weight_decay=wd, serial=serial)
+        p = torch.tensor(x0[0], dtype=torch.float64, requires_grad=True)
+        opt = torch.optim.SGD([p], lr=lr, momentum=mu, weight_decay=wd)
+        for k in range(iters):
+            p.grad = torch.tensor(G[k, 0], dtype=torch.float64)
+            opt.step()
+            # serial: version k is replaced by what the worker sent, x'_k = x_k - lr d_k (= the optimiser's state)
+            np.testing.assert_allclose(X[(0, k)] if serial else X[(0, k + 1)], p.detach().numpy(), atol=1e-12)
+        np.testing.assert_allclose(X[(0, iters)], p.detach().numpy(), atol=1e-12)
+
+
+@pytest.mark.parametrize("n_in", [inputs.ring(5), inputs.torus(3, 3), inputs.complete(4)])
+def test_serial_approach_is_apply_then_average(n_in):
+    # serial approach of Section 3.2 with equal speeds: X_{k+1} = W^T (X_k - lr G_k)
+    rng = np.random.default_rng(13)
+    N, C, iters, lr = len(n_in), 7, 5, 0.2
+    x0 = rng.standard_normal((N, C))
+    G = rng.standard_normal((iters, N, C))
+    tr = trace_equal_speed(n_in, iters)
+    X, _ = up.run_updates(tr, N, lr, 0.0, x0, up.GradExternal(G), keep_all=True, serial=True)
+    W = uniform_W(n_in)
+    Xk = x0.copy()
+    for k in range(iters):
+        sent = Xk - lr * G[k]
+        for i in range(N):
+            np.testing.assert_allclose(X[(i, k)], sent[i], atol=1e-12)        # version k as sent
+        Xk = W.T @ sent
+    for i in range(N):
+        np.testing.assert_allclose(X[(i, iters)], Xk[i], atol=1e-12)
+    # and it differs from the parallel approach as soon as replicas differ
+    Xp, _ = up.run_updates(tr, N, lr, 0.0, x0, up.GradExternal(G), keep_all=True)
+    assert np.abs(Xp[(0, iters)] - X[(0, iters)]).max() > 1e-3
