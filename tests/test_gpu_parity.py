@@ -421,3 +421,46 @@ def test_unsupported_combinations_are_refused():
         g.h.step()
     assert e.value.code == hop.E_UNSUPPORTED
     g.h.close()
+
+
+def test_tensor_path_with_more_than_eight_ring_slots_and_few_workers():
+    # s + 1 = 10 slots: no output tensor map per slot is kept, rows leave by bulk copies; N = 24 < 32 workers
+    N, P, iters, s = 24, 128 * 5, 14, 9
+    ptr, idx = inputs.graph_to_csr(inputs.complete(N))
+    rng = np.random.default_rng(9)
+    w = inputs.Workload(0, "dense-deep-ring", N, P, iters, s=s, b=3, max_skip=0, max_ig=9, lr=0.05, momentum=0.0,
+                        weight_mode=inputs.STALE_LINEAR, grad_mode=inputs.GRAD_SYNTHETIC, in_ptr=ptr, in_idx=idx,
+                        ticks=rng.choice([1, 2, 9], size=(N, iters)).astype(np.uint64), grad_seed=99)
+    w._p0 = rng.standard_normal(P).astype(np.float32)
+    g = GpuRun(w, hop.MIX_TENSOR)
+    assert all(g.h.level_stats(k)["kernel"] == hop.MIX_TENSOR for k in range(iters))
+    assert max(g.h.level_stats(k)["U"] for k in range(iters)) > N          # stale versions really are consumed
+    g.h.close()
+    check(w, iters, TOL_RUN, hop.MIX_TENSOR, perturb=True)
+
+
+def test_streaming_rejects_bad_records_and_run_checks_its_range():
+    w = inputs.make_workload(4, P=256, iters=6)
+    g = GpuRun(w)
+    tr = g.trace.to_arrays()
+    N = w.N
+    a, b = tr["ptr"][0], tr["ptr"][N]
+    good = [np.ascontiguousarray(tr["op"][0]), (tr["ptr"][:N + 1] - a).astype(np.int64), np.ascontiguousarray(tr["nbr"][a:b]),
+            np.ascontiguousarray(tr["ver"][a:b]), np.ascontiguousarray(tr["num"][a:b]), np.ascontiguousarray(tr["den"][0])]
+    bad = [x.copy() for x in good]
+    bad[3][2] = 5                                      # a version from the future
+    g.h.set_level(0)
+    with pytest.raises(hop.HopError) as e:
+        g.h.step_host(*bad)
+    assert e.value.code == hop.E_TRACE
+    g.h.step_host(*good)                               # the rejected call left the context usable
+    g.h.set_level(0)
+    g.h.run(0)
+    with pytest.raises(hop.HopError) as e:
+        g.h.run(w.iters + 1)
+    assert e.value.code == hop.E_STATE
+    g.h.run(w.iters)
+    with pytest.raises(hop.HopError):
+        g.h.step()
+    assert g.h.read_status() == 0
+    g.h.close()
