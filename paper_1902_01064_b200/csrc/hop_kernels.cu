@@ -1,9 +1,11 @@
 // CUDA kernels of the Hop hot path for sm_100a.
 //
 //   mix_staged / mix_bulk   fused Recv-Reduce-Apply for one level: x_{k+1,i} = sum w * x_{v,j} - lr * d
-//                           (Fig. alg0 steps 2-3, Reduce of Fig. alg4 / Eq. 2), SGD or momentum
+//                           (Fig. alg0 steps 2-3, Reduce of Fig. alg4 / Eq. 2), SGD or momentum, weight decay
 //   synth_grad              G[i][p] = sigma * normal(seed, i, k, p)
-//   svm_margin_* / svm_dense_grad / svm_csr_apply   hinge-loss linear SVM gradient and sparse Apply
+//   svm_margin_* / svm_dense_grad / svm_csr_apply   hinge- or log-loss linear model gradient and sparse Apply
+//   apply_dense             serial approach (Section 3.2): x_k <- x_k - lr * d before the level's Reduce
+// (the dense-graph tensor-core kernel lives in hop_dense_tc.cu)
 //
 // In-place ring: version k+1 of a worker overwrites the slot of version k-s, which other workers may
 // consume in the same level.  A thread block therefore owns a column tile for ALL workers: it first
