@@ -209,9 +209,10 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
     }
     __syncthreads();
     if (warp < kProducerWarps) {
-        // ---------------- producers: this warp issues rows warp*32 + lane, + 32*kProducerWarps, ...
-        int my_rows = 0;
-        for (int r0 = warp * 32; r0 < rows; r0 += 32 * kProducerWarps) my_rows += min(32, rows - r0);
+        // ---------------- producers: row r goes to warp r % kProducerWarps, lane (r / kProducerWarps) % 32, so that
+        // every warp issues the same number of copies (+-1): a warp issues them one after the other, ~30-40 ns
+        // each, and the busiest warp sets the pace (measured)
+        const int my_rows = (rows - warp + kProducerWarps - 1) / kProducerWarps;
         int64_t n = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++n) {
@@ -224,7 +225,7 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
             if (lane == 0) mbar_expect_tx(&full[s], bytes * (uint32_t)my_rows);
             __syncwarp();
             float* dst = stage0 + s * stage_floats;
-            for (int r = warp * 32 + lane; r < rows; r += 32 * kProducerWarps) {
+            for (int r = warp + lane * kProducerWarps; r < rows; r += 32 * kProducerWarps) {
                 const float* src;
                 if (r < lv.U) src = X + (int64_t)lv.src_row[r] * P;
                 else if (r < lv.U + nG) src = G + (int64_t)lv.grad_workers[r - lv.U] * P;
