@@ -188,6 +188,15 @@ int hop_set_level(hop_ctx* ctx, int32_t level);
  * then the fused gather-mix-update writing slot k+1, then (CSR SVM) the sparse apply.
  * Asynchronous; HOP_E_STATE past the end of the trace. */
 int hop_step(hop_ctx* ctx);
+/* Split-phase form of hop_step for a parameter vector sharded by columns over several contexts (one per GPU):
+ * mixing and the dense / synthetic gradients are separable by column, but an SVM margin a_r . x needs all columns.
+ * hop_step_begin enqueues the gradient phase; in the SVM modes it stops after the partial margins over this
+ * context's columns and returns their device address (double[N * batch], owned by the context; entry
+ * [i * batch + r] for row r of worker i's minibatch) for the caller to sum across the shards -- e.g. one NCCL
+ * all-reduce on the bound stream.  hop_step_end computes the coefficients from the summed margins and finishes the
+ * level.  With one shard, begin + end equals hop_step.  In the other gradient modes *margins is NULL, *count 0. */
+int hop_step_begin(hop_ctx* ctx, double** margins, int64_t* count);
+int hop_step_end(hop_ctx* ctx);
 /* Executes the next n_levels levels of the loaded trace.  When the bound stream is not the default
  * stream, the levels are captured once into a CUDA graph (cached per (first level, n_levels); dropped
  * by any bind / option / trace change) and replayed, which removes most of the per-kernel launch cost

@@ -35,6 +35,8 @@ struct hop_ctx {
     const int32_t* svmCol = nullptr;
     int32_t svmR = 0, svmB = 0;
     float* coef = nullptr;
+    double* margins = nullptr;       // [N][batch] margins of the current minibatches (split-phase stepping)
+    bool mid_step = false;           // hop_step_begin done, hop_step_end pending
     // loaded trace (owned device tables)
     std::vector<HopLevelHost> levels;
     float* d_tcw = nullptr;         // tensor-core path: weight numerators, row tables, padded slice rows
@@ -138,12 +140,14 @@ static void free_trace_tables(hop_ctx* c) {
     c->d_tcw = nullptr; c->d_tcrows = nullptr; c->d_tcsrc = nullptr;
     c->levels.clear();
     c->loaded = false;
+    c->mid_step = false;
 }
 
 extern "C" int hop_destroy(hop_ctx* c) {
     if (!c) return HOP_OK;
     free_trace_tables(c);
     if (c->coef) cudaFree(c->coef);
+    if (c->margins) cudaFree(c->margins);
     if (c->d_err) cudaFree(c->d_err);
     if (c->d_stage) cudaFree(c->d_stage);
     if (c->h_stage) cudaFreeHost(c->h_stage);
@@ -250,7 +254,10 @@ static int alloc_coef(hop_ctx* c, int32_t R, int32_t B) {
     const int rc = ensure_device(c);
     if (rc) return rc;
     if (c->coef) { cudaFree(c->coef); c->coef = nullptr; }
+    if (c->margins) { cudaFree(c->margins); c->margins = nullptr; }
     HOP_CUDA(c, cudaMalloc(&c->coef, (size_t)c->g.N * B * sizeof(float)));
+    HOP_CUDA(c, cudaMalloc(&c->margins, (size_t)c->g.N * B * sizeof(double)));
+    HOP_CUDA(c, cudaMemset(c->margins, 0, (size_t)c->g.N * B * sizeof(double)));
     c->svmR = R; c->svmB = B;
     return HOP_OK;
 }
@@ -389,6 +396,7 @@ extern "C" int hop_load_trace(hop_ctx* c, const hop_trace* t) {
     c->levels = std::move(levels);
     c->sent = std::move(sent);
     c->loaded = true;
+    c->mid_step = false;
     c->level = 0;
     std::fill(c->newest.begin(), c->newest.end(), 0);
     return HOP_OK;
@@ -433,7 +441,9 @@ static int ensure_tc_maps(hop_ctx* c) {
     return HOP_OK;
 }
 
-static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, const TcPtrs& tc) {
+// phase 0: the whole level.  phase 1: the gradient phase only (SVM modes stop after the partial margins).
+// phase 2: the rest (SVM modes start from the margins the caller has summed over the column shards).
+static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, const TcPtrs& tc, int phase = 0) {
     size_t t0 = 0, t1 = 0;
     HopLaunchCfg cfg{};
     cfg.X = c->X; cfg.M = c->M; cfg.G = c->G; cfg.P = c->P; cfg.N = c->g.N; cfg.s = c->s;
@@ -446,16 +456,20 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, c
         HOP_SPAN_BEGIN();
         switch (c->grad_mode) {
         case HOP_GRAD_SYNTHETIC:
-            e = hop_launch_synth_grad(cfg, lv, c->grad_seed, (float)c->sigma, c->col_offset); c->launches += 1; break;
+            if (phase != 2) { e = hop_launch_synth_grad(cfg, lv, c->grad_seed, (float)c->sigma, c->col_offset); c->launches += 1; }
+            break;
         case HOP_GRAD_SVM_DENSE:
-            e = hop_launch_svm_dense(cfg, lv, c->svmA, c->svmY, c->svmR, c->svmB, c->coef); c->launches += 2; break;
+            e = hop_launch_svm_dense(cfg, lv, c->svmA, c->svmY, c->svmR, c->svmB, c->coef, c->margins, phase);
+            c->launches += phase == 1 ? 1 : 2; break;
         case HOP_GRAD_SVM_CSR:
-            e = hop_launch_svm_csr_coef(cfg, lv, c->svmRowPtr, c->svmCol, c->svmVal, c->svmY, c->svmR, c->svmB, c->coef); c->launches += 1; break;
+            e = hop_launch_svm_csr_coef(cfg, lv, c->svmRowPtr, c->svmCol, c->svmVal, c->svmY, c->svmR, c->svmB, c->coef, c->margins, phase);
+            c->launches += 1; break;
         default: break;
         }
         if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("gradient kernel launch: ") + cudaGetErrorString((cudaError_t)e));
         HOP_SPAN_END(0, 0);
     }
+    if (phase == 1) return HOP_OK;
     if (c->serial && L.nG > 0) {      // Apply on x_k before it is sent: dense update kernel, or the sparse apply on slot k
         HOP_SPAN_BEGIN();
         if (c->grad_mode == HOP_GRAD_SVM_CSR)
@@ -489,8 +503,42 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, c
     return HOP_OK;
 }
 
+static int step_phase(hop_ctx* c, int phase) {
+    if (!c->bound || !c->loaded) HOP_FAIL(c, HOP_E_STATE, "hop_step_begin/end: bind buffers and load a trace first");
+    if (c->level >= (int32_t)c->levels.size()) HOP_FAIL(c, HOP_E_STATE, "hop_step_begin/end: past the end of the trace");
+    if ((phase == 1) == c->mid_step) HOP_FAIL(c, HOP_E_STATE, "hop_step_begin and hop_step_end must alternate");
+    int rc = check_mode(c);
+    if (rc) return rc;
+    const HopLevelHost& L = c->levels[c->level];
+    HopLevelDev lv{c->d_i32 + L.off_src, c->d_rec + L.off_rec, c->d_ent + L.off_ent, c->d_i32 + L.off_gw, L.U, L.nA, L.nG, c->level};
+    rc = run_level(c, L, lv, TcPtrs{c->d_tcw + L.off_tcw, c->d_tcrows + L.off_tcrows, c->d_tcsrc + L.off_tcsrc}, phase);
+    if (rc) return rc;
+    c->mid_step = phase == 1;
+    if (phase == 2) {
+        for (const HopRecord& r : L.recs) c->newest[r.worker] = c->level + 1;
+        c->level += 1;
+    }
+    return HOP_OK;
+}
+
+extern "C" int hop_step_begin(hop_ctx* c, double** margins, int64_t* count) {
+    if (!c) return HOP_E_ARG;
+    const int rc = step_phase(c, 1);
+    if (rc) return rc;
+    const bool svm = c->grad_mode == HOP_GRAD_SVM_DENSE || c->grad_mode == HOP_GRAD_SVM_CSR;
+    if (margins) *margins = svm ? c->margins : nullptr;
+    if (count) *count = svm ? (int64_t)c->g.N * c->svmB : 0;
+    return HOP_OK;
+}
+
+extern "C" int hop_step_end(hop_ctx* c) {
+    if (!c) return HOP_E_ARG;
+    return step_phase(c, 2);
+}
+
 extern "C" int hop_step(hop_ctx* c) {
     if (!c) return HOP_E_ARG;
+    if (c->mid_step) HOP_FAIL(c, HOP_E_STATE, "hop_step: a hop_step_begin is waiting for its hop_step_end");
     if (!c->bound || !c->loaded) HOP_FAIL(c, HOP_E_STATE, "hop_step: bind buffers and load a trace first");
     if (c->level >= (int32_t)c->levels.size()) HOP_FAIL(c, HOP_E_STATE, "hop_step: past the end of the trace");
     int rc = check_mode(c);
@@ -514,6 +562,7 @@ static int enqueue_level(hop_ctx* c, int32_t k) {
 extern "C" int hop_run(hop_ctx* c, int32_t n_levels) {
     if (!c) return HOP_E_ARG;
     if (!c->bound || !c->loaded) HOP_FAIL(c, HOP_E_STATE, "hop_run: bind buffers and load a trace first");
+    if (c->mid_step) HOP_FAIL(c, HOP_E_STATE, "hop_run: a hop_step_begin is waiting for its hop_step_end");
     if (n_levels < 0 || c->level + n_levels > (int32_t)c->levels.size()) HOP_FAIL(c, HOP_E_STATE, "hop_run: past the end of the trace");
     if (n_levels == 0) return HOP_OK;
     int rc = check_mode(c);
@@ -558,6 +607,7 @@ extern "C" int hop_step_host(hop_ctx* c, const int32_t* op, const int64_t* ptr, 
     if (!c) return HOP_E_ARG;
     if (!op || !ptr || !den) HOP_FAIL(c, HOP_E_ARG, "hop_step_host: null pointer");
     if (!c->bound) HOP_FAIL(c, HOP_E_STATE, "hop_step_host: bind buffers first");
+    if (c->mid_step) HOP_FAIL(c, HOP_E_STATE, "hop_step_host: a hop_step_begin is waiting for its hop_step_end");
     if (probe_len < 0 || probe_len > c->P) HOP_FAIL(c, HOP_E_ARG, "hop_step_host: probe_len out of range");
     int rc = check_mode(c);
     if (rc) return rc;
@@ -628,6 +678,7 @@ extern "C" int hop_step_host(hop_ctx* c, const int32_t* op, const int64_t* ptr, 
 extern "C" int hop_set_level(hop_ctx* c, int32_t level) {
     if (!c) return HOP_E_ARG;
     if (level < 0 || (c->loaded && level > (int32_t)c->levels.size())) HOP_FAIL(c, HOP_E_ARG, "hop_set_level: out of range");
+    c->mid_step = false;
     // newest version held by each worker after levels [0, level)
     std::fill(c->newest.begin(), c->newest.end(), 0);
     if (c->loaded)

@@ -129,10 +129,11 @@ struct HopLaunchCfg {
 int hop_launch_mix_staged(const HopLaunchCfg& c, const HopLevelDev& lv);
 int hop_launch_mix_bulk(const HopLaunchCfg& c, const HopLevelDev& lv);
 int hop_launch_synth_grad(const HopLaunchCfg& c, const HopLevelDev& lv, uint64_t seed, float sigma, int64_t col_offset);
+// phase 0 = whole gradient; 1 = partial margins into `margins` only; 2 = coefficients from `margins`, then the rest
 int hop_launch_svm_dense(const HopLaunchCfg& c, const HopLevelDev& lv, const float* A, const float* y,
-                         int32_t R, int32_t B, float* coef);
+                         int32_t R, int32_t B, float* coef, double* margins, int phase);
 int hop_launch_svm_csr_coef(const HopLaunchCfg& c, const HopLevelDev& lv, const int64_t* row_ptr, const int32_t* col,
-                            const float* val, const float* y, int32_t R, int32_t B, float* coef);
+                            const float* val, const float* y, int32_t R, int32_t B, float* coef, double* margins, int phase);
 // slot_shift 1: apply to x_{k+1} after the mix (parallel approach); 0: to x_k before it (serial approach)
 int hop_launch_svm_csr_apply(const HopLaunchCfg& c, const HopLevelDev& lv, const int64_t* row_ptr, const int32_t* col,
                              const float* val, int32_t R, int32_t B, const float* coef, int32_t slot_shift);

@@ -339,7 +339,7 @@ __device__ __forceinline__ float loss_coefficient(float y, double m, int B, int 
 __global__ void __launch_bounds__(256)
 svm_margin_csr_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelDev lv, const int64_t* __restrict__ row_ptr,
                       const int32_t* __restrict__ col, const float* __restrict__ val, const float* __restrict__ y,
-                      int R, int B, int loss, float* __restrict__ coef) {
+                      int R, int B, int loss, float* __restrict__ coef, double* __restrict__ margins_out) {
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (gw >= lv.nG * B) return;
     const int a = gw / B, r = gw - a * B;
@@ -349,12 +349,28 @@ svm_margin_csr_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelDev
     double m = 0.0;
     for (int64_t t = row_ptr[row] + lane; t < row_ptr[row + 1]; t += 32) m += (double)val[t] * (double)x[col[t]];
     m = warp_sum(m);
-    if (lane == 0) coef[(int64_t)worker * B + r] = loss_coefficient(y[row], m, B, loss);
+    if (lane == 0) {
+        if (margins_out) margins_out[(int64_t)worker * B + r] = m;     // partial margin over this shard's columns
+        else coef[(int64_t)worker * B + r] = loss_coefficient(y[row], m, B, loss);
+    }
+}
+
+// Coefficients from margins that were summed over column shards (one thread per minibatch row).
+__global__ void __launch_bounds__(256)
+svm_coef_from_margins_kernel(const double* __restrict__ margins, HopLevelDev lv, const float* __restrict__ y, int R, int B,
+                             int loss, float* __restrict__ coef) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= lv.nG * B) return;
+    const int a = t / B, r = t - a * B;
+    const int worker = lv.grad_workers[a];
+    const int64_t row = (int64_t)worker * R + (int64_t)(lv.level % (R / B)) * B + r;
+    coef[(int64_t)worker * B + r] = loss_coefficient(y[row], margins[(int64_t)worker * B + r], B, loss);
 }
 
 __global__ void __launch_bounds__(256)
 svm_margin_dense_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelDev lv, const float* __restrict__ A,
-                        const float* __restrict__ y, int R, int B, int loss, float* __restrict__ coef) {
+                        const float* __restrict__ y, int R, int B, int loss, float* __restrict__ coef,
+                        double* __restrict__ margins_out) {
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (gw >= lv.nG * B) return;
     const int a = gw / B, r = gw - a * B;
@@ -365,7 +381,10 @@ svm_margin_dense_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelD
     double m = 0.0;
     for (int64_t p = lane; p < P; p += 32) m += (double)arow[p] * (double)x[p];
     m = warp_sum(m);
-    if (lane == 0) coef[(int64_t)worker * B + r] = loss_coefficient(y[row], m, B, loss);
+    if (lane == 0) {
+        if (margins_out) margins_out[(int64_t)worker * B + r] = m;
+        else coef[(int64_t)worker * B + r] = loss_coefficient(y[row], m, B, loss);
+    }
 }
 
 // g[i][p] = sum_r coef_r * A[r][p]; one thread per column, rows of the minibatch in order.
@@ -504,23 +523,35 @@ int hop_launch_synth_grad(const HopLaunchCfg& c, const HopLevelDev& lv, uint64_t
     return (int)cudaGetLastError();
 }
 
+// phase 0: margins, coefficients (and the dense gradient) in one go.  phase 1: only the partial margins over this
+// context's columns, written to `margins`.  phase 2: coefficients from the (summed) margins, then the dense gradient.
 int hop_launch_svm_dense(const HopLaunchCfg& c, const HopLevelDev& lv, const float* A, const float* y,
-                         int32_t R, int32_t B, float* coef) {
+                         int32_t R, int32_t B, float* coef, double* margins, int phase) {
     if (lv.nG == 0) return 0;
     const int warps = lv.nG * B;
-    svm_margin_dense_kernel<<<(warps * 32 + 255) / 256, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.P, c.s + 1, lv, A, y, R, B, c.loss, coef);
+    cudaStream_t st = (cudaStream_t)c.stream;
+    if (phase != 2)
+        svm_margin_dense_kernel<<<(warps * 32 + 255) / 256, 256, 0, st>>>(c.X, c.P, c.s + 1, lv, A, y, R, B, c.loss, coef,
+                                                                          phase == 1 ? margins : nullptr);
+    if (phase == 1) return (int)cudaGetLastError();
+    if (phase == 2) svm_coef_from_margins_kernel<<<(warps + 255) / 256, 256, 0, st>>>(margins, lv, y, R, B, c.loss, coef);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return (int)e;
     dim3 grid((unsigned)((c.P + 255) / 256), (unsigned)lv.nG);
-    svm_dense_grad_kernel<<<grid, 256, 0, (cudaStream_t)c.stream>>>(c.G, c.P, lv, A, R, B, coef);
+    svm_dense_grad_kernel<<<grid, 256, 0, st>>>(c.G, c.P, lv, A, R, B, coef);
     return (int)cudaGetLastError();
 }
 
 int hop_launch_svm_csr_coef(const HopLaunchCfg& c, const HopLevelDev& lv, const int64_t* row_ptr, const int32_t* col,
-                            const float* val, const float* y, int32_t R, int32_t B, float* coef) {
+                            const float* val, const float* y, int32_t R, int32_t B, float* coef, double* margins, int phase) {
     if (lv.nG == 0) return 0;
     const int warps = lv.nG * B;
-    svm_margin_csr_kernel<<<(warps * 32 + 255) / 256, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.P, c.s + 1, lv, row_ptr, col, val, y, R, B, c.loss, coef);
+    cudaStream_t st = (cudaStream_t)c.stream;
+    if (phase != 2)
+        svm_margin_csr_kernel<<<(warps * 32 + 255) / 256, 256, 0, st>>>(c.X, c.P, c.s + 1, lv, row_ptr, col, val, y, R, B, c.loss, coef,
+                                                                        phase == 1 ? margins : nullptr);
+    else
+        svm_coef_from_margins_kernel<<<(warps + 255) / 256, 256, 0, st>>>(margins, lv, y, R, B, c.loss, coef);
     return (int)cudaGetLastError();
 }
 

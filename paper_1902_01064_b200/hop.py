@@ -51,6 +51,8 @@ SIGNATURES = {
     "hop_set_level": [_p, _i32],
     "hop_step": [_p],
     "hop_run": [_p, _i32],
+    "hop_step_begin": [_p, C.POINTER(_p), C.POINTER(_i64)],
+    "hop_step_end": [_p],
     "hop_step_host": [_p, _p, _p, _p, _p, _p, _p, _p, _i64],
     "hop_read_status": [_p, C.POINTER(_i32)],
     "hop_level_stats": [_p, _i32, _p],
@@ -63,6 +65,14 @@ for _name, _args in SIGNATURES.items():
     _f = getattr(lib, _name)
     _f.argtypes = _args
     _f.restype = C.c_char_p if _name == "hop_last_error" else C.c_int
+
+
+class DeviceSpan:
+    """A context-owned run of device memory, described through the CUDA array interface so that
+    torch.as_tensor(span, device=...) wraps it without a copy (for a collective on it)."""
+
+    def __init__(self, ptr: int, count: int, typestr: str = "<f8"):
+        self.__cuda_array_interface__ = {"shape": (count,), "typestr": typestr, "data": (ptr, False), "version": 3}
 
 
 class HopError(RuntimeError):
@@ -184,6 +194,15 @@ class Hop:
 
     def step(self):
         self._chk(lib.hop_step(self.h))
+
+    def step_begin(self):
+        """Returns (device address of the partial margins, count of doubles); (None, 0) outside the SVM modes."""
+        ptr, n = _p(), _i64()
+        self._chk(lib.hop_step_begin(self.h, C.byref(ptr), C.byref(n)))
+        return ptr.value, n.value
+
+    def step_end(self):
+        self._chk(lib.hop_step_end(self.h))
 
     def run(self, n_levels):
         self._chk(lib.hop_run(self.h, n_levels))

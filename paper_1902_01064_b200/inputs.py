@@ -161,6 +161,15 @@ class SvmData:
     col: Optional[np.ndarray] = None       # [nnz] int32
     val: Optional[np.ndarray] = None       # [nnz] float32
 
+    def column_shard(self, lo: int, hi: int) -> "SvmData":
+        """The features with index in [lo, hi), renumbered from 0: what one rank of a column-sharded run binds."""
+        if self.dense is not None:
+            return SvmData(self.rows_per_worker, self.batch, self.y, dense=np.ascontiguousarray(self.dense[..., lo:hi]))
+        keep = (self.col >= lo) & (self.col < hi)
+        kept_before = np.concatenate([[0], np.cumsum(keep, dtype=np.int64)])
+        return SvmData(self.rows_per_worker, self.batch, self.y, row_ptr=kept_before[self.row_ptr],
+                       col=(self.col[keep] - lo).astype(np.int32), val=self.val[keep])
+
 
 @dataclass
 class Workload:

@@ -464,3 +464,60 @@ def test_streaming_rejects_bad_records_and_run_checks_its_range():
         g.h.step()
     assert g.h.read_status() == 0
     g.h.close()
+
+
+# ------------------------------------------------------------------ column-sharded SVM: split-phase stepping
+@pytest.mark.parametrize("cfg,P,iters,edges", [(1, 1000, 40, (0, 384, 1000)), (2, 4096, 24, (0, 1024, 2560, 4096))])
+def test_column_sharded_svm_with_summed_margins_equals_the_oracle(cfg, P, iters, edges):
+    """Each shard owns a column range (its own context, ring and feature slice); the partial margins are summed
+    between hop_step_begin and hop_step_end, as an all-reduce would between ranks.  Shards run one after the other
+    on one stream, so nothing waits on anything."""
+    import dataclasses
+    w = inputs.make_workload(cfg, P=P, iters=iters)
+    x0 = np.stack([w.p0() + w.perturbation(i) for i in range(w.N)])
+    shards = []
+    for lo, hi in zip(edges, edges[1:]):
+        ws = dataclasses.replace(w, P=hi - lo, svm=w.svm.column_shard(lo, hi), _p0=None)
+        shards.append(GpuRun(ws, x0=np.ascontiguousarray(x0[:, lo:hi])))
+    for k in range(iters):
+        views = []
+        for g in shards:
+            ptr, n = g.h.step_begin()
+            assert n == w.N * w.svm.batch and ptr
+            views.append((ptr, n))
+        # plumbing: wrap the context-owned buffers and sum them in place (what dist.all_reduce does across ranks)
+        bufs = [_as_f64_tensor(ptr, n) for ptr, n in views]
+        total = torch.stack(bufs).sum(0)
+        for b in bufs:
+            b.copy_(total)
+        for g in shards:
+            g.h.step_end()
+    tr, want, newest = oracle_run(w, x0, iters)
+    scale = max(np.abs(x).max() for x in want)
+    worst = 0.0
+    for g, lo, hi in zip(shards, edges, edges[1:]):
+        assert g.h.read_status() == 0
+        for i in range(w.N):
+            assert g.h.newest_version(i) == newest[i]
+            worst = max(worst, np.abs(g.h.read_params(i).astype(np.float64) - want[i][lo:hi]).max())
+        g.h.close()
+    assert worst <= TOL_RUN * scale, (worst, scale)
+
+
+def _as_f64_tensor(ptr, n):
+    return torch.as_tensor(hop.DeviceSpan(ptr, n), device=DEV)
+
+
+def test_split_phase_calls_must_alternate():
+    w = inputs.make_workload(1, P=256, iters=8)
+    g = GpuRun(w)
+    with pytest.raises(hop.HopError):
+        g.h.step_end()
+    g.h.step_begin()
+    for call in (g.h.step_begin, g.h.step, lambda: g.h.run(1)):
+        with pytest.raises(hop.HopError):
+            call()
+    g.h.step_end()
+    g.h.step()
+    assert g.h.read_status() == 0
+    g.h.close()

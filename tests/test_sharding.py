@@ -68,3 +68,46 @@ def test_two_ranks_reproduce_the_unsharded_run(tmp_path):
     X, newest = up.run_updates(tr, w.N, w.lr, w.momentum, x0, up.GradSynthetic(w.grad_seed, w.sigma, np.arange(P)), s=w.s)
     want = np.stack([X[(i, newest[i])] for i in range(w.N)])
     assert np.array_equal(got, want)
+
+
+def _dense_rows(svm, P):
+    """Every worker's rows as one dense [N*R][P] float64 matrix, whichever layout the data has."""
+    if svm.dense is not None:
+        return svm.dense.reshape(-1, P).astype(np.float64)
+    A = np.zeros((len(svm.row_ptr) - 1, P))
+    for r in range(len(svm.row_ptr) - 1):
+        a, b = svm.row_ptr[r], svm.row_ptr[r + 1]
+        np.add.at(A[r], svm.col[a:b], svm.val[a:b])
+    return A
+
+
+@pytest.mark.parametrize("cfg,P", [(1, 1000), (2, 2048)])
+def test_feature_column_shards_partition_the_data(cfg, P):
+    w = inputs.make_workload(cfg, P=P, iters=4)
+    full = _dense_rows(w.svm, P)
+    edges = (0, 128, 896, P)
+    parts = [_dense_rows(w.svm.column_shard(lo, hi), hi - lo) for lo, hi in zip(edges, edges[1:])]
+    assert np.array_equal(np.concatenate(parts, axis=1), full)
+
+
+def _margin_rank(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    P = 2048
+    w = inputs.make_workload(2, P=P, iters=4)
+    lo, hi = bench.shard_columns(P, world, rank)
+    x = w.p0().astype(np.float64)[lo:hi]
+    part = torch.from_numpy(_dense_rows(w.svm.column_shard(lo, hi), hi - lo) @ x)     # this rank's partial margins
+    dist.all_reduce(part)                                                             # the one exchange step of an SVM level
+    if rank == 0:
+        np.save(out, part.numpy())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_partial_margins_summed_over_two_ranks_equal_the_full_margins(tmp_path):
+    out = str(tmp_path / "margins.npy")
+    mp.spawn(_margin_rank, args=(2, _free_port(), out), nprocs=2, join=True)
+    w = inputs.make_workload(2, P=2048, iters=4)
+    want = _dense_rows(w.svm, 2048) @ w.p0().astype(np.float64)
+    assert np.allclose(np.load(out), want, rtol=1e-12, atol=1e-12)
