@@ -213,6 +213,20 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
         // every warp issues the same number of copies (+-1): a warp issues them one after the other, ~30-40 ns
         // each, and the busiest warp sets the pace (measured)
         const int my_rows = (rows - warp + kProducerWarps - 1) / kProducerWarps;
+        // a lane's rows are the same for every tile: the first kHoist source addresses are formed once (the row
+        // tables are in global memory; reading them per tile would put a global-load latency before every copy)
+        constexpr int kHoist = 2;
+        auto row_src = [&](int r) -> const float* {
+            if (r < lv.U) return X + (int64_t)lv.src_row[r] * P;
+            if (r < lv.U + nG) return G + (int64_t)lv.grad_workers[r - lv.U] * P;
+            return M + (int64_t)lv.grad_workers[r - lv.U - nG] * P;
+        };
+        const float* src_h[kHoist];
+#pragma unroll
+        for (int h = 0; h < kHoist; ++h) {
+            const int r = warp + (lane + 32 * h) * kProducerWarps;
+            src_h[h] = r < rows ? row_src(r) : nullptr;
+        }
         int64_t n = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++n) {
@@ -225,13 +239,11 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
             if (lane == 0) mbar_expect_tx(&full[s], bytes * (uint32_t)my_rows);
             __syncwarp();
             float* dst = stage0 + s * stage_floats;
-            for (int r = warp + lane * kProducerWarps; r < rows; r += 32 * kProducerWarps) {
-                const float* src;
-                if (r < lv.U) src = X + (int64_t)lv.src_row[r] * P;
-                else if (r < lv.U + nG) src = G + (int64_t)lv.grad_workers[r - lv.U] * P;
-                else src = M + (int64_t)lv.grad_workers[r - lv.U - nG] * P;
-                bulk_g2s(dst + (int64_t)r * w, src + c0, bytes, &full[s]);
-            }
+#pragma unroll
+            for (int h = 0; h < kHoist; ++h)
+                if (src_h[h]) bulk_g2s(dst + (warp + (lane + 32 * h) * kProducerWarps) * w, src_h[h] + c0, bytes, &full[s]);
+            for (int r = warp + (lane + 32 * kHoist) * kProducerWarps; r < rows; r += 32 * kProducerWarps)
+                bulk_g2s(dst + (int64_t)r * w, row_src(r) + c0, bytes, &full[s]);
         }
         // drain: do not leave while copies into this block's shared memory are still in flight
         if (ok) {
