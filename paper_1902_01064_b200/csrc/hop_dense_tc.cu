@@ -135,8 +135,10 @@ struct TcSmem {                       // control block at the start of dynamic s
     int epi_fail;
     uint32_t active_mask[4], g_mask[4];   // bit i of word i/32: worker i writes a result / applies a gradient
     alignas(16) float inv_den[128];
+    alignas(16) int32_t src[256];         // ring row of each of the K consumed slices (read by the producers for every chunk)
     HopTcRow rows[128];
 };
+static_assert(sizeof(TcSmem) <= 4096, "control block");
 
 __global__ void __launch_bounds__(kThreads, 1)
 mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapG,
@@ -164,6 +166,7 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     for (int i = tid; i < 128; i += kThreads) { cb->rows[i] = tbl[i]; cb->inv_den[i] = tbl[i].inv_den; }
+    for (int i = tid; i < Kpad; i += kThreads) cb->src[i] = src_row[i];
     if (tid < 4) {
         uint32_t am = 0, gm = 0;
         for (int i = 0; i < 32; ++i) { am |= (uint32_t)(tbl[tid * 32 + i].out_row >= 0) << i; gm |= (uint32_t)(tbl[tid * 32 + i].g_row >= 0) << i; }
@@ -198,8 +201,9 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                 if (lane < 2) {
                     const int r4 = half * 2 + lane;                 // which group of four rows of the chunk
                     const int u = c * kChunk + r4 * 4;
+                    const int4 rows4 = *reinterpret_cast<const int4*>(&cb->src[u]);
                     tma_gather4(raw + (size_t)s * (kChunk * kTile) + r4 * 4 * kTile, &mapX, (int)(tile * kTile),
-                                src_row[u], src_row[u + 1], src_row[u + 2], src_row[u + 3], &cb->raw_full[s]);
+                                rows4.x, rows4.y, rows4.z, rows4.w, &cb->raw_full[s]);
                 }
                 if (++s == raw_stages) { s = 0; ph ^= 1u; }
             }
