@@ -486,7 +486,7 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, c
         if (L.kernel == HOP_MIX_TENSOR)
             e = hop_launch_mix_dense_tc(cfg, c->tc_mapX, c->tc_mapG,
                                         (L.nA == c->g.N && c->tc_slots > 0) ? c->tc_mapY + 128 * ((lv.level + 1) % (c->s + 1)) : nullptr,
-                                        tc.w, tc.rows, tc.src, L.Kpad);
+                                        tc.w, tc.rows, tc.src, L.Kpad, L.tc_rows.data());
         else
             e = (L.kernel == HOP_MIX_BULK) ? hop_launch_mix_bulk(cfg, lv) : hop_launch_mix_staged(cfg, lv);
         c->launches += 1;

@@ -15,12 +15,13 @@
 //               of the ring per instruction), two per warp: a warp issues at ~27 ns per row fetched (measured)
 //   warp 1      MMA issue (one elected lane): tcgen05.mma kind::tf32, M=128 (columns) x N=128 (workers) x K=8,
 //               A operand (X_hi / X_lo) from tensor memory, B operand (A^T, resident) from shared memory
-//   warp 3      gradient producer: one 2-D TMA box load of the tile's N x 128 piece of G into shared memory
-//   warps 4-7   converters: lane = column; read the raw chunk from shared memory, split hi/lo with
-//               round-to-nearest TF32 splitting, tcgen05.st into the A stages in tensor memory
-//   warps 8-11  epilogue: tcgen05.ld both accumulators, add, release them, then y = acc/den - lr*g written over g
-//               in shared memory; the finished N x 128 tile goes to the output slot as one TMA box store (or
-//               one bulk row copy per active worker when some workers are idle in the level)
+//   warp 3      gradient loader and result storer: the tile's N x 128 piece of G comes in, and the finished results
+//               leave, in quarters of 32 workers (2-D TMA boxes; one bulk row copy per active worker when some
+//               workers are idle in the level); a quarter is refilled as soon as its results have been read out
+//   warps 4-11  converters, two groups taking alternate chunks: lane = column; read the raw chunk from shared
+//               memory, split hi/lo with round-to-nearest TF32 splitting, tcgen05.st into the A stages
+//   warps 12-19 epilogue, two groups owning 64 workers each: tcgen05.ld both accumulators, add, release them, then
+//               y = acc/den - lr*g written over g in shared memory, quarter by quarter
 // Tensor memory (512 columns): D_hi 0..127, D_lo 128..255, eight A stages of 32 columns (hi 16 + lo 16).
 // Shared memory: control block, A^T (Kpad x 512 B), the G tile (64 KB), 3..8 raw stages of 8 KB.
 // Every wait is bounded; a time-out sets the error word and lets the block run to its normal exit,
@@ -31,6 +32,7 @@
 #include <algorithm>
 #include <cstdint>
 #include <cstring>
+#include <type_traits>
 
 #include "hop_internal.h"
 
@@ -39,7 +41,7 @@ namespace {
 constexpr int kTile = 128;          // parameter columns per tile = MMA M
 constexpr int kChunk = 16;          // K rows per pipeline stage
 constexpr int kStages = 8;          // tensor-memory A stages (power of two); raw shared-memory stages: 3..8, chosen by the host
-constexpr int kThreads = 12 * 32;
+constexpr int kThreads = 20 * 32;
 constexpr uint32_t kSpin = 1u << 20;
 constexpr int kRawStageBytes = kChunk * kTile * 4;          // 8 KB
 constexpr int kGTileBytes = 128 * kTile * 4;                // 64 KB
@@ -127,14 +129,33 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// Per-worker constants of a level, passed by value: the epilogue is fully unrolled over the workers, so each use is
+// a constant-bank operand at a fixed offset instead of a shared-memory load.
+// 16 columns of both accumulators for this thread's lane, added: one wait for the two loads.
+__device__ __forceinline__ void tmem_ld16_sum(uint32_t t_hi, uint32_t t_lo, float* out) {
+    uint32_t h[16], l[16];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3]), "=r"(h[4]), "=r"(h[5]), "=r"(h[6]), "=r"(h[7]), "=r"(h[8]), "=r"(h[9]),
+                   "=r"(h[10]), "=r"(h[11]), "=r"(h[12]), "=r"(h[13]), "=r"(h[14]), "=r"(h[15]) : "r"(t_hi) : "memory");
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(l[0]), "=r"(l[1]), "=r"(l[2]), "=r"(l[3]), "=r"(l[4]), "=r"(l[5]), "=r"(l[6]), "=r"(l[7]), "=r"(l[8]), "=r"(l[9]),
+                   "=r"(l[10]), "=r"(l[11]), "=r"(l[12]), "=r"(l[13]), "=r"(l[14]), "=r"(l[15]) : "r"(t_lo) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) out[i] = __uint_as_float(h[i]) + __uint_as_float(l[i]);
+}
+
+struct TcRowConsts {
+    float inv_den[128];                  // 1 / (sum of the worker's integer weights)
+    uint32_t active_mask[4], g_mask[4];  // bit i of word i/32: worker i writes a result / applies a gradient
+};
+
 struct TcSmem {                       // control block at the start of dynamic shared memory
     uint64_t raw_full[kStages], raw_empty[kStages], a_full[kStages], a_empty[kStages];
-    uint64_t acc_full, acc_empty, w_full, g_full, g_empty;
+    uint64_t acc_full, acc_empty, w_full;
+    uint64_t g_full[4], y_full[4];        // one pair per quarter (32 workers) of the gradient / result tile
     uint32_t tmem_base;
     int abort_flag;
-    int epi_fail;
-    uint32_t active_mask[4], g_mask[4];   // bit i of word i/32: worker i writes a result / applies a gradient
-    alignas(16) float inv_den[128];
     alignas(16) int32_t src[256];         // ring row of each of the K consumed slices (read by the producers for every chunk)
     HopTcRow rows[128];
 };
@@ -145,7 +166,7 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                     const __grid_constant__ CUtensorMap mapY, int box_store,
                     float* __restrict__ X, int64_t P, int n_workers, float lr, const float* __restrict__ Wk,
                     const HopTcRow* __restrict__ tbl, const int32_t* __restrict__ src_row, int Kpad, int raw_stages,
-                    int32_t* __restrict__ err_word) {
+                    int32_t* __restrict__ err_word, const __grid_constant__ TcRowConsts rc) {
     extern __shared__ __align__(1024) unsigned char smem[];
     TcSmem* cb = reinterpret_cast<TcSmem*>(smem);
     float* Wsm = reinterpret_cast<float*>(smem + 4096);                        // Kpad * 512 bytes, canonical K-major
@@ -158,20 +179,14 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mb_init(&cb->raw_full[s], 2); mb_init(&cb->raw_empty[s], 4); mb_init(&cb->a_full[s], 4); mb_init(&cb->a_empty[s], 1); }
-        mb_init(&cb->acc_full, 1); mb_init(&cb->acc_empty, 4); mb_init(&cb->w_full, 1);
-        mb_init(&cb->g_full, 1); mb_init(&cb->g_empty, 1);
+        mb_init(&cb->acc_full, 1); mb_init(&cb->acc_empty, 8); mb_init(&cb->w_full, 1);
+        for (int q = 0; q < 4; ++q) { mb_init(&cb->g_full[q], 1); mb_init(&cb->y_full[q], 4); }
         cb->abort_flag = 0;
-        cb->epi_fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    for (int i = tid; i < 128; i += kThreads) { cb->rows[i] = tbl[i]; cb->inv_den[i] = tbl[i].inv_den; }
+    for (int i = tid; i < 128; i += kThreads) cb->rows[i] = tbl[i];
     for (int i = tid; i < Kpad; i += kThreads) cb->src[i] = src_row[i];
-    if (tid < 4) {
-        uint32_t am = 0, gm = 0;
-        for (int i = 0; i < 32; ++i) { am |= (uint32_t)(tbl[tid * 32 + i].out_row >= 0) << i; gm |= (uint32_t)(tbl[tid * 32 + i].g_row >= 0) << i; }
-        cb->active_mask[tid] = am; cb->g_mask[tid] = gm;
-    }
     if (warp == 2) {   // tensor-memory allocation: all 512 columns, by one warp, which also frees them
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(s32(&cb->tmem_base)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -239,29 +254,65 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             if (!ok) { atomicCAS(err_word, 0, ERR_TC_WAIT | 2); cb->abort_flag = 1; }
         }
     } else if (warp == 3) {
-        // ------------------------------------------------ gradient tile producer
-        int n_rows = 0;
-        for (int i = 0; i < 128; ++i) n_rows += (cb->rows[i].g_row >= 0);
+        // ------------------------------------------------ gradient loader and result storer.  The gradient / result
+        // tile is handled in quarters of 32 workers: g_full[q] tells the epilogue that quarter q holds the gradients
+        // of its tile, y_full[q] tells this warp that the results have replaced them.  This warp then sends the
+        // quarter out, waits until the copy engine has read it, and refills it with the next tile's gradients, so
+        // the epilogue warps never wait for a store (as one chain load -> compute -> store took 4.4 of 5.8 us per
+        // tile, measured).  Without gradients the refill is a plain arrival: g_full then only says "free".
+        const bool has_g = (rc.g_mask[0] | rc.g_mask[1] | rc.g_mask[2] | rc.g_mask[3]) != 0;
+        const int nq = (n_workers + 31) / 32;
+        const uint32_t qbytes = (uint32_t)min(32, n_workers) * kTile * 4u;      // the box of the map; rows out of range arrive as zeros
+        auto refill = [&](int q, int64_t tile) {
+            if (has_g) {
+                mb_expect_tx(&cb->g_full[q], qbytes);
+                tma_tile2d(Gsm + q * 32 * kTile, &mapG, (int)(tile * kTile), q * 32, &cb->g_full[q]);
+            } else {
+                mb_arrive(&cb->g_full[q]);
+            }
+        };
+        if (lane == 0 && (int64_t)blockIdx.x < tiles)
+            for (int q = 0; q < nq; ++q) refill(q, blockIdx.x);
         int64_t tcount = 0;
         bool ok = true;
-        if (n_rows > 0)
-            for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++tcount) {
-                if (!mb_wait(&cb->g_empty, (uint32_t)((tcount & 1) ^ 1), abort_flag)) { ok = false; break; }
-                if (lane == 0) {      // rows 0..n_workers-1 of G, columns of this tile, in one box
-                    mb_expect_tx(&cb->g_full, (uint32_t)n_workers * kTile * 4u);
-                    tma_tile2d(Gsm, &mapG, (int)(tile * kTile), 0, &cb->g_full);
+        for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
+            for (int q = 0; q < nq; ++q) {
+                if (!mb_wait(&cb->y_full[q], (uint32_t)(tcount & 1), abort_flag)) { ok = false; break; }
+                if (box_store) {
+                    if (lane == 0) {   // all workers active: one box [32 workers x 128] into the output slot
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                                     ::"l"(&mapY), "r"((int)(tile * kTile)), "r"(q * 32), "r"(s32(Gsm + q * 32 * kTile)) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    }
+                } else {               // one 512-byte row copy per active worker of the quarter
+                    const HopTcRow rw = cb->rows[q * 32 + lane];
+                    if (rw.out_row >= 0) {
+                        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                                     ::"l"(X + (int64_t)rw.out_row * P + tile * kTile), "r"(s32(Gsm + (q * 32 + lane) * kTile)), "r"(kTile * 4) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    }
                 }
-                __syncwarp();
+                __syncwarp();          // the quarter has been read out of shared memory
+                if (lane == 0 && tile + gridDim.x < tiles) refill(q, tile + gridDim.x);
             }
+        }
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // this thread's stores have reached global memory
         if (!ok && lane == 0) { atomicCAS(err_word, 0, ERR_TC_WAIT | 5); cb->abort_flag = 1; }
-    } else if (warp >= 4 && warp < 8) {
-        // ------------------------------------------------ converters (lane quarter = warp % 4)
-        const int col = (warp - 4) * 32 + lane;
+    } else if (warp >= 4 && warp < 12) {
+        // ------------------------------------------------ converters (lane quarter = warp % 4): two groups of four
+        // warps, the first takes the even chunks, the second the odd ones (a chunk's tensor-memory stage has the
+        // chunk's parity, kStages being even).  With one group the converter warps, at one busy warp per scheduler,
+        // ran at ~0.2 instructions per cycle and set the pace of the block (measured).
+        const int par = (warp - 4) >> 2;
+        const int col = ((warp - 4) & 3) * 32 + lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        int64_t q = 0;
+        const int64_t my_tiles = (int64_t)blockIdx.x < tiles ? (tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+        const int64_t total = my_tiles * nchunks;
         bool ok = true;
-        // The tensor-memory store of chunk q is left in flight while chunk q+1 is fetched from shared memory;
-        // chunk q is published to the MMA warp (a_full) once tcgen05.wait::st has covered it.
+        // The tensor-memory store of a chunk is left in flight while this warp's next chunk is fetched from shared
+        // memory; the chunk is published to the MMA warp (a_full) once tcgen05.wait::st has covered it.
         int pending = -1;
         auto publish = [&]() {
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -270,116 +321,101 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             if (lane == 0) mb_arrive(&cb->a_full[pending]);
             pending = -1;
         };
-        int rs = 0;
+        int rs = par;              // raw stage of chunk q and its phase bit, advanced by hand (3 <= raw_stages <= 8)
         uint32_t rph = 0;
-        for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
-            for (int c = 0; c < nchunks; ++c, ++q) {
-                const int s = (int)(q & (kStages - 1));
-                if (pending >= 0 && !mb_try(&cb->raw_full[rs], rph)) publish();   // nothing to overlap with
-                if (!mb_wait(&cb->raw_full[rs], rph, abort_flag)) { ok = false; break; }
-                const float* r = raw + (size_t)rs * (kChunk * kTile) + col;
-                float x[kChunk];
+        for (int64_t q = par; q < total; q += 2) {
+            const int s = (int)(q & (kStages - 1));
+            // With an odd number of raw stages a stage alternates between the two groups, and this group may get here
+            // before the other one has even seen the stage's previous chunk: the parity test on raw_full would then
+            // pass on that older phase.  So first make sure the previous chunk of the stage has been released.
+            if (pending >= 0 && !(mb_try(&cb->raw_empty[rs], rph ^ 1u) && mb_try(&cb->raw_full[rs], rph))) publish();   // nothing to overlap with
+            if (!mb_wait(&cb->raw_empty[rs], rph ^ 1u, abort_flag)) { ok = false; break; }
+            if (!mb_wait(&cb->raw_full[rs], rph, abort_flag)) { ok = false; break; }
+            const float* r = raw + (size_t)rs * (kChunk * kTile) + col;
+            float x[kChunk];
 #pragma unroll
-                for (int u = 0; u < kChunk; ++u) x[u] = r[u * kTile];
-                if (pending >= 0) publish();
-                if (!mb_wait(&cb->a_empty[s], (uint32_t)(((q / kStages) & 1) ^ 1), abort_flag)) { ok = false; break; }
-                fence_after();
-                uint32_t v[2 * kChunk];                      // hi in columns 0..15 of the stage, lo in 16..31
+            for (int u = 0; u < kChunk; ++u) x[u] = r[u * kTile];
+            if (pending >= 0) publish();
+            if (!mb_wait(&cb->a_empty[s], (uint32_t)(((q / kStages) & 1) ^ 1), abort_flag)) { ok = false; break; }
+            fence_after();
+            uint32_t v[2 * kChunk];                      // hi in columns 0..15 of the stage, lo in 16..31
 #pragma unroll
-                for (int u = 0; u < kChunk; ++u) {
-                    v[u] = to_tf32(x[u]);
-                    v[kChunk + u] = to_tf32(x[u] - __uint_as_float(v[u]));
-                }
-                __syncwarp();
-                if (lane == 0) mb_arrive(&cb->raw_empty[rs]);   // the raw chunk is in registers
-                tmem_st32(tmem + lane_base + kA0 + s * 32, v);
-                pending = s;
-                if (++rs == raw_stages) { rs = 0; rph ^= 1u; }
+            for (int u = 0; u < kChunk; ++u) {
+                v[u] = to_tf32(x[u]);
+                v[kChunk + u] = to_tf32(x[u] - __uint_as_float(v[u]));
             }
+            __syncwarp();
+            if (lane == 0) mb_arrive(&cb->raw_empty[rs]);   // the raw chunk is in registers
+            tmem_st32(tmem + lane_base + kA0 + s * 32, v);
+            pending = s;
+            rs += 2;
+            if (rs >= raw_stages) { rs -= raw_stages; rph ^= 1u; }
         }
         if (pending >= 0) publish();
         if (!ok && lane == 0) { atomicCAS(err_word, 0, ERR_TC_WAIT | 3); cb->abort_flag = 1; }
-    } else if (warp >= 8) {
-        // ------------------------------------------------ epilogue (lane quarter = warp % 4)
-        const int col = (warp - 8) * 32 + lane;
+    } else if (warp >= 12) {
+        // ------------------------------------------------ epilogue (lane quarter = warp % 4): two groups of four warps,
+        // the first owns workers 0..63 (quarters 0, 1 of the tile), the second workers 64..127 (quarters 2, 3)
+        const int col = ((warp - 12) & 3) * 32 + lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        uint32_t am[4], gm[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) { am[k] = cb->active_mask[k]; gm[k] = cb->g_mask[k]; }
-        const bool has_g = (gm[0] | gm[1] | gm[2] | gm[3]) != 0;
-        int64_t tcount = 0;
-        bool ok = true;
-        for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++tcount) {
-            // A warp whose wait times out still walks through both named barriers of the iteration and
-            // raises epi_fail, so that all four epilogue warps leave the loop together.
-            bool fail = !mb_wait(&cb->acc_full, (uint32_t)(tcount & 1), abort_flag);
-            if (!fail) {
+        const int nq = (n_workers + 31) / 32;
+        auto run = [&](auto half_c) {
+            constexpr int H = decltype(half_c)::value;      // compile-time, so that every per-worker constant is an immediate offset
+            int64_t tcount = 0;
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
+                if (!mb_wait(&cb->acc_full, (uint32_t)(tcount & 1), abort_flag)) { ok = false; break; }
                 fence_after();
-                float acc[128];
+                float acc[64];
+                if (H * 2 < nq) {
 #pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    float h[32], l[32];
-                    tmem_ld32(tmem + lane_base + kDhi + b * 32, h);
-                    tmem_ld32(tmem + lane_base + kDlo + b * 32, l);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) acc[b * 32 + i] = h[i] + l[i];
+                    for (int j = 0; j < 4; ++j) tmem_ld16_sum(tmem + lane_base + kDhi + H * 64 + j * 16, tmem + lane_base + kDlo + H * 64 + j * 16, acc + j * 16);
                 }
                 fence_before();
                 __syncwarp();
                 if (lane == 0) mb_arrive(&cb->acc_empty);   // the next tile's MMAs may overwrite the accumulators now
-                fail = has_g && !mb_wait(&cb->g_full, (uint32_t)(tcount & 1), abort_flag);
-                if (!fail) {
-                    // y = acc/den - lr*g replaces g in the shared tile (column-per-thread: conflict-free), then the
-                    // tile leaves through the copy engine: per-thread 4-byte global stores of 128 different rows
-                    // were the slowest part of the kernel by far (measured)
-                    // Batches of 8 rows with every shared-memory load ahead of the batch's stores: the compiler
-                    // cannot prove that the stores do not alias the tables, and a load-store-load chain per row
-                    // cost ~100 cycles per row (measured).
+                // y = acc/den - lr*g replaces g in the shared tile (column-per-thread: conflict-free), then the tile
+                // leaves through the copy engine: per-thread 4-byte global stores of 128 different rows were the
+                // slowest part of the kernel by far (measured).
 #pragma unroll
-                    for (int b = 0; b < 128; b += 8) {
-                        const float4 s0 = *reinterpret_cast<const float4*>(&cb->inv_den[b]);
-                        const float4 s1 = *reinterpret_cast<const float4*>(&cb->inv_den[b + 4]);
-                        const float sc[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-                        float g[8];
+                for (int qq = 0; qq < 2; ++qq) {
+                    const int q = H * 2 + qq;
+                    if (q < nq && ok) {
+                        if (!mb_wait(&cb->g_full[q], (uint32_t)(tcount & 1), abort_flag)) { ok = false; }
+                        else {
+                            // Batches of 8 rows, the gradients of the next batch fetched before the stores of this
+                            // one: the compiler cannot prove that the stores do not alias later loads, and a
+                            // load-store-load chain per row cost ~100 cycles per row (measured).
+                            float g[8], gn[8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) g[i] = Gsm[(b + i) * kTile + col];   // stale but unused when the row has no gradient
+                            for (int i = 0; i < 8; ++i) g[i] = Gsm[(q * 32 + i) * kTile + col];   // stale but unused when the row has no gradient
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const int r = b + i;
-                            const float gv = ((gm[r >> 5] >> (r & 31)) & 1u) ? g[i] : 0.f;
-                            if ((am[r >> 5] >> (r & 31)) & 1u) Gsm[r * kTile + col] = fmaf(-lr, gv, acc[r] * sc[i]);
+                            for (int b = 0; b < 32; b += 8) {
+                                if (b + 8 < 32) {
+#pragma unroll
+                                    for (int i = 0; i < 8; ++i) gn[i] = Gsm[(q * 32 + b + 8 + i) * kTile + col];
+                                }
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    const int r = (H * 2 + qq) * 32 + b + i;           // worker
+                                    const float gv = ((rc.g_mask[r >> 5] >> (r & 31)) & 1u) ? g[i] : 0.f;
+                                    if ((rc.active_mask[r >> 5] >> (r & 31)) & 1u)
+                                        Gsm[r * kTile + col] = fmaf(-lr, gv, acc[qq * 32 + b + i] * rc.inv_den[r]);
+                                }
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) g[i] = gn[i];
+                            }
+                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // results visible to the copy engine
+                            __syncwarp();
+                            if (lane == 0) mb_arrive(&cb->y_full[q]);
                         }
                     }
                 }
             }
-            if (fail) *((volatile int*)&cb->epi_fail) = 1;
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            const bool any_fail = *((volatile int*)&cb->epi_fail) != 0;
-            if (!any_fail) {
-                if (box_store) {
-                    if (warp == 8 && lane == 0) {  // all workers active: one box [n_workers x 128] into the output slot
-                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-                                     ::"l"(&mapY), "r"((int)(tile * kTile)), "r"(0), "r"(s32(Gsm)) : "memory");
-                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                    }
-                } else {                           // one 512-byte row copy per active worker
-                    const int e = tid - 8 * 32;
-                    const HopTcRow rw = cb->rows[e];
-                    if (rw.out_row >= 0) {
-                        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                                     ::"l"(X + (int64_t)rw.out_row * P + tile * kTile), "r"(s32(Gsm + e * kTile)), "r"(kTile * 4) : "memory");
-                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                    }
-                }
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");   // the tile has been read out of shared memory
-            if (any_fail) { ok = false; break; }
-            if (has_g && warp == 8 && lane == 0) mb_arrive(&cb->g_empty);    // the next tile's gradient rows may land now
-        }
-        if (!ok && lane == 0) { atomicCAS(err_word, 0, ERR_TC_WAIT | 4); cb->abort_flag = 1; }
+            if (!ok && lane == 0) { atomicCAS(err_word, 0, ERR_TC_WAIT | 4); cb->abort_flag = 1; }
+        };
+        if (warp < 16) run(std::integral_constant<int, 0>{});
+        else run(std::integral_constant<int, 1>{});
     }
     fence_before();
     __syncthreads();
@@ -399,10 +435,10 @@ size_t hop_dense_tc_smem(int Kpad) {
 }
 
 // Tensor maps: X as [N*(s+1) rows][P] with a one-row box of 128 columns (the tile::gather4 form loads four
-// such rows), G as [N rows][P] with an N x 128 box.  cuTensorMapEncodeTiled is looked up through the
+// such rows), G as [N rows][P] with a min(32, N) x 128 box (one quarter of a tile).  cuTensorMapEncodeTiled is looked up through the
 // runtime so that the library does not link against the driver.
 // mapY[slot]: the rows {i*(s+1) + slot} of X, i.e. the output slot of a level, as an [N rows][P] tensor with row
-// stride (s+1)*P and an N x 128 box (n_slots maps of 128 bytes each).
+// stride (s+1)*P and the same box as G (n_slots maps of 128 bytes each).
 int hop_dense_tc_make_maps(float* X, int64_t ring_rows, const float* G, int32_t N, int64_t P, void* mapX, void* mapG,
                            void* mapY, int32_t n_slots) {
     typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -431,7 +467,7 @@ int hop_dense_tc_make_maps(float* X, int64_t ring_rows, const float* G, int32_t 
     if (G) {
         const cuuint64_t dims[2] = {(cuuint64_t)P, (cuuint64_t)N};
         const cuuint64_t strides[1] = {(cuuint64_t)P * 4};
-        const cuuint32_t box[2] = {(cuuint32_t)kTile, (cuuint32_t)N};
+        const cuuint32_t box[2] = {(cuuint32_t)kTile, (cuuint32_t)std::min(32, N)};
         if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(G), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                    CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return (int)cudaErrorInvalidValue;
@@ -441,7 +477,7 @@ int hop_dense_tc_make_maps(float* X, int64_t ring_rows, const float* G, int32_t 
     for (int slot = 0; slot < n_slots; ++slot) {
         const cuuint64_t dims[2] = {(cuuint64_t)P, (cuuint64_t)N};
         const cuuint64_t strides[1] = {(cuuint64_t)S * P * 4};
-        const cuuint32_t box[2] = {(cuuint32_t)kTile, (cuuint32_t)N};
+        const cuuint32_t box[2] = {(cuuint32_t)kTile, (cuuint32_t)std::min(32, N)};
         if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, X + (int64_t)slot * P, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                    CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return (int)cudaErrorInvalidValue;
@@ -451,17 +487,23 @@ int hop_dense_tc_make_maps(float* X, int64_t ring_rows, const float* G, int32_t 
 }
 
 int hop_launch_mix_dense_tc(const HopLaunchCfg& c, const void* mapX, const void* mapG, const void* mapY, const float* Wk,
-                            const HopTcRow* tbl, const int32_t* src_row, int Kpad) {
+                            const HopTcRow* tbl, const int32_t* src_row, int Kpad, const HopTcRow* host_rows) {
     alignas(64) CUtensorMap mx, mg, my;
     std::memcpy(&mx, mapX, sizeof(mx));
     std::memcpy(&mg, mapG, sizeof(mg));
     std::memcpy(&my, mapY ? mapY : mapX, sizeof(my));
+    TcRowConsts rc{};
+    for (int i = 0; i < 128; ++i) {
+        rc.inv_den[i] = host_rows[i].inv_den;
+        rc.active_mask[i >> 5] |= (uint32_t)(host_rows[i].out_row >= 0) << (i & 31);
+        rc.g_mask[i >> 5] |= (uint32_t)(host_rows[i].g_row >= 0) << (i & 31);
+    }
     const size_t smem = hop_dense_tc_smem(Kpad);
     cudaError_t e = hop_allow_max_smem<mix_dense_tc_kernel>();
     if (e != cudaSuccess) return (int)e;
     const int64_t tiles = c.P / kTile;
     const int grid = (int)std::min<int64_t>(tiles, (int64_t)c.sm_count);
     mix_dense_tc_kernel<<<grid, kThreads, smem, (cudaStream_t)c.stream>>>(mx, mg, my, mapY ? 1 : 0, c.X, c.P, c.N, c.lr, Wk, tbl, src_row, Kpad,
-                                                                          raw_stages_for(Kpad), c.err_word);
+                                                                          raw_stages_for(Kpad), c.err_word, rc);
     return (int)cudaGetLastError();
 }

@@ -146,6 +146,7 @@ int hop_mix_table_limit();
 size_t hop_dense_tc_smem(int Kpad);
 int hop_dense_tc_make_maps(float* X, int64_t ring_rows, const float* G, int32_t N, int64_t P, void* mapX, void* mapG,
                            void* mapY, int32_t n_slots);   // 128-byte blobs; mapY holds n_slots of them
-// mapY = the output slot's map when every worker is active in the level, else nullptr (row-by-row stores)
+// mapY = the output slot's map when every worker is active in the level, else nullptr (row-by-row stores);
+// host_rows = the host copy of tbl (its per-worker constants travel as kernel parameters)
 int hop_launch_mix_dense_tc(const HopLaunchCfg& c, const void* mapX, const void* mapG, const void* mapY, const float* Wk,
-                            const HopTcRow* tbl, const int32_t* src_row, int Kpad);
+                            const HopTcRow* tbl, const int32_t* src_row, int Kpad, const HopTcRow* host_rows);

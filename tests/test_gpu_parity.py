@@ -439,6 +439,23 @@ def test_tensor_path_with_more_than_eight_ring_slots_and_few_workers():
     check(w, iters, TOL_RUN, hop.MIX_TENSOR, perturb=True)
 
 
+def test_tensor_path_with_a_ragged_last_quarter_of_workers():
+    # N = 40: the second quarter of the gradient / result tile holds 8 real workers; the copy engine zero-fills the
+    # rows past N on the way in and drops them on the way out
+    N, P, iters, s = 40, 128 * 7, 10, 1
+    ptr, idx = inputs.graph_to_csr(inputs.complete(N))
+    rng = np.random.default_rng(11)
+    w = inputs.Workload(0, "dense-40", N, P, iters, s=s, b=4, max_skip=0, max_ig=1, lr=0.05, momentum=0.0,
+                        weight_mode=inputs.STALE_LINEAR, grad_mode=inputs.GRAD_SYNTHETIC, in_ptr=ptr, in_idx=idx,
+                        ticks=rng.choice([1, 2, 5], size=(N, iters)).astype(np.uint64), grad_seed=77)
+    w._p0 = rng.standard_normal(P).astype(np.float32)
+    g = GpuRun(w, hop.MIX_TENSOR)
+    assert all(g.h.level_stats(k)["kernel"] == hop.MIX_TENSOR for k in range(iters))
+    g.h.close()
+    check(w, iters, TOL_RUN, hop.MIX_TENSOR, perturb=True)
+    check(w, 1, TOL_STEP, hop.MIX_TENSOR, perturb=True)
+
+
 def test_streaming_rejects_bad_records_and_run_checks_its_range():
     w = inputs.make_workload(4, P=256, iters=6)
     g = GpuRun(w)
