@@ -32,7 +32,6 @@
 #include <algorithm>
 #include <cstdint>
 #include <cstring>
-#include <type_traits>
 
 #include "hop_internal.h"
 
@@ -355,67 +354,82 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         if (!ok && lane == 0) { atomicCAS(err_word, 0, ERR_TC_WAIT | 3); cb->abort_flag = 1; }
     } else if (warp >= 12) {
         // ------------------------------------------------ epilogue (lane quarter = warp % 4): two groups of four warps,
-        // the first owns workers 0..63 (quarters 0, 1 of the tile), the second workers 64..127 (quarters 2, 3)
+        // the first owns workers 0..63 (quarters 0, 1 of the tile), the second workers 64..127 (quarters 2, 3).
+        // The loop over the workers has to be unrolled (the accumulators are registers), and the unrolled code is
+        // what every tile streams through the instruction cache: one copy serves both groups (the group only
+        // moves base addresses), and the usual quarter, where every worker is active and has a gradient, has a
+        // body without the mask tests.
+        const int half = (warp - 12) >> 2;
         const int col = ((warp - 12) & 3) * 32 + lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const int nq = (n_workers + 31) / 32;
-        auto run = [&](auto half_c) {
-            constexpr int H = decltype(half_c)::value;      // compile-time, so that every per-worker constant is an immediate offset
-            int64_t tcount = 0;
-            bool ok = true;
-            for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
-                if (!mb_wait(&cb->acc_full, (uint32_t)(tcount & 1), abort_flag)) { ok = false; break; }
-                fence_after();
-                float acc[64];
-                if (H * 2 < nq) {
+        int64_t tcount = 0;
+        bool ok = true;
+        for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
+            if (!mb_wait(&cb->acc_full, (uint32_t)(tcount & 1), abort_flag)) { ok = false; break; }
+            fence_after();
+            float acc[64];
+            if (half * 2 < nq) {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) tmem_ld16_sum(tmem + lane_base + kDhi + H * 64 + j * 16, tmem + lane_base + kDlo + H * 64 + j * 16, acc + j * 16);
-                }
-                fence_before();
-                __syncwarp();
-                if (lane == 0) mb_arrive(&cb->acc_empty);   // the next tile's MMAs may overwrite the accumulators now
-                // y = acc/den - lr*g replaces g in the shared tile (column-per-thread: conflict-free), then the tile
-                // leaves through the copy engine: per-thread 4-byte global stores of 128 different rows were the
-                // slowest part of the kernel by far (measured).
+                for (int j = 0; j < 4; ++j) tmem_ld16_sum(tmem + lane_base + kDhi + half * 64 + j * 16, tmem + lane_base + kDlo + half * 64 + j * 16, acc + j * 16);
+            }
+            fence_before();
+            __syncwarp();
+            if (lane == 0) mb_arrive(&cb->acc_empty);   // the next tile's MMAs may overwrite the accumulators now
+            // y = acc/den - lr*g replaces g in the shared tile (column-per-thread: conflict-free), then the tile leaves
+            // through the copy engine: per-thread 4-byte global stores of 128 different rows were the slowest part of
+            // the kernel by far (measured).
 #pragma unroll
-                for (int qq = 0; qq < 2; ++qq) {
-                    const int q = H * 2 + qq;
-                    if (q < nq && ok) {
-                        if (!mb_wait(&cb->g_full[q], (uint32_t)(tcount & 1), abort_flag)) { ok = false; }
-                        else {
-                            // Batches of 8 rows, the gradients of the next batch fetched before the stores of this
-                            // one: the compiler cannot prove that the stores do not alias later loads, and a
-                            // load-store-load chain per row cost ~100 cycles per row (measured).
-                            float g[8], gn[8];
+            for (int qq = 0; qq < 2; ++qq) {
+                const int q = half * 2 + qq;
+                if (q < nq && ok) {
+                    if (!mb_wait(&cb->g_full[q], (uint32_t)(tcount & 1), abort_flag)) { ok = false; }
+                    else {
+                        float* Gq = Gsm + q * 32 * kTile + col;
+                        const float* dq = rc.inv_den + q * 32;
+                        const uint32_t amq = rc.active_mask[q], gmq = rc.g_mask[q];
+                        // Batches of 8 rows, the gradients of the next batch fetched before the stores of this one:
+                        // the compiler cannot prove that the stores do not alias later loads, and a load-store-load
+                        // chain per row cost ~100 cycles per row (measured).
+                        float g[8], gn[8];
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) g[i] = Gsm[(q * 32 + i) * kTile + col];   // stale but unused when the row has no gradient
+                        for (int i = 0; i < 8; ++i) g[i] = Gq[i * kTile];   // stale but unused when the row has no gradient
+                        if (amq == 0xffffffffu && gmq == 0xffffffffu) {
 #pragma unroll
                             for (int b = 0; b < 32; b += 8) {
                                 if (b + 8 < 32) {
 #pragma unroll
-                                    for (int i = 0; i < 8; ++i) gn[i] = Gsm[(q * 32 + b + 8 + i) * kTile + col];
+                                    for (int i = 0; i < 8; ++i) gn[i] = Gq[(b + 8 + i) * kTile];
+                                }
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) Gq[(b + i) * kTile] = fmaf(-lr, g[i], acc[qq * 32 + b + i] * dq[b + i]);
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) g[i] = gn[i];
+                            }
+                        } else {
+#pragma unroll
+                            for (int b = 0; b < 32; b += 8) {
+                                if (b + 8 < 32) {
+#pragma unroll
+                                    for (int i = 0; i < 8; ++i) gn[i] = Gq[(b + 8 + i) * kTile];
                                 }
 #pragma unroll
                                 for (int i = 0; i < 8; ++i) {
-                                    const int r = (H * 2 + qq) * 32 + b + i;           // worker
-                                    const float gv = ((rc.g_mask[r >> 5] >> (r & 31)) & 1u) ? g[i] : 0.f;
-                                    if ((rc.active_mask[r >> 5] >> (r & 31)) & 1u)
-                                        Gsm[r * kTile + col] = fmaf(-lr, gv, acc[qq * 32 + b + i] * rc.inv_den[r]);
+                                    const float gv = ((gmq >> (b + i)) & 1u) ? g[i] : 0.f;
+                                    if ((amq >> (b + i)) & 1u) Gq[(b + i) * kTile] = fmaf(-lr, gv, acc[qq * 32 + b + i] * dq[b + i]);
                                 }
 #pragma unroll
                                 for (int i = 0; i < 8; ++i) g[i] = gn[i];
                             }
-                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // results visible to the copy engine
-                            __syncwarp();
-                            if (lane == 0) mb_arrive(&cb->y_full[q]);
                         }
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // results visible to the copy engine
+                        __syncwarp();
+                        if (lane == 0) mb_arrive(&cb->y_full[q]);
                     }
                 }
             }
-            if (!ok && lane == 0) { atomicCAS(err_word, 0, ERR_TC_WAIT | 4); cb->abort_flag = 1; }
-        };
-        if (warp < 16) run(std::integral_constant<int, 0>{});
-        else run(std::integral_constant<int, 1>{});
+        }
+        if (!ok && lane == 0) { atomicCAS(err_word, 0, ERR_TC_WAIT | 4); cb->abort_flag = 1; }
     }
     fence_before();
     __syncthreads();
