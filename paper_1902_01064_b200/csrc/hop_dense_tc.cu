@@ -22,7 +22,7 @@
 //               memory, split hi/lo with round-to-nearest TF32 splitting, tcgen05.st into the A stages
 //   warps 12-19 epilogue, two groups owning 64 workers each: tcgen05.ld both accumulators, add, release them, then
 //               y = acc/den - lr*g written over g in shared memory, quarter by quarter
-// Tensor memory (512 columns): D_hi 0..127, D_lo 128..255, eight A stages of 32 columns (hi 16 + lo 16).
+// Tensor memory (512 columns): D_hi 0..127, D_lo 128..255, four A stages of 64 columns (two chunks of hi 16 + lo 16).
 // Shared memory: control block, A^T (Kpad x 512 B), the G tile (64 KB), 3..8 raw stages of 8 KB.
 // Every wait is bounded; a time-out sets the error word and lets the block run to its normal exit,
 // where tensor memory is released.
@@ -39,7 +39,8 @@ namespace {
 
 constexpr int kTile = 128;          // parameter columns per tile = MMA M
 constexpr int kChunk = 16;          // K rows per pipeline stage
-constexpr int kStages = 8;          // tensor-memory A stages (power of two); raw shared-memory stages: 3..8, chosen by the host
+constexpr int kStages = 8;          // most raw shared-memory stages (3..8, chosen by the host)
+constexpr int kAStages = 4;         // tensor-memory A stages of two chunks each (one per converter group)
 constexpr int kThreads = 20 * 32;
 constexpr uint32_t kSpin = 1u << 20;
 constexpr int kRawStageBytes = kChunk * kTile * 4;          // 8 KB
@@ -177,7 +178,7 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
     volatile int* abort_flag = &cb->abort_flag;
 
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) { mb_init(&cb->raw_full[s], 2); mb_init(&cb->raw_empty[s], 4); mb_init(&cb->a_full[s], 4); mb_init(&cb->a_empty[s], 1); }
+        for (int s = 0; s < kStages; ++s) { mb_init(&cb->raw_full[s], 2); mb_init(&cb->raw_empty[s], 4); mb_init(&cb->a_full[s], 8); mb_init(&cb->a_empty[s], 1); }
         mb_init(&cb->acc_full, 1); mb_init(&cb->acc_empty, 8); mb_init(&cb->w_full, 1);
         for (int q = 0; q < 4; ++q) { mb_init(&cb->g_full[q], 1); mb_init(&cb->y_full[q], 4); }
         cb->abort_flag = 0;
@@ -232,18 +233,24 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
                 if (!mb_wait(&cb->acc_empty, (uint32_t)((tcount & 1) ^ 1), abort_flag)) { ok = false; break; }
                 fence_after();
-                for (int c = 0; c < nchunks; ++c, ++q) {
-                    const int s = (int)(q % kStages);
-                    if (!mb_wait(&cb->a_full[s], (uint32_t)((q / kStages) & 1), abort_flag)) { ok = false; break; }
+                // One wait, fence and commit per pair of chunks: waiting, fencing and committing cost this thread
+                // more than the four MMAs of a chunk take on the tensor pipe (measured), and this thread sets the
+                // pace of the main loop.
+                for (int c = 0; c < nchunks; c += 2, ++q) {
+                    const int s = (int)(q % kAStages);
+                    if (!mb_wait(&cb->a_full[s], (uint32_t)((q / kAStages) & 1), abort_flag)) { ok = false; break; }
                     fence_after();
-                    const uint32_t a_hi = tmem + kA0 + s * 32, a_lo = a_hi + 16;
 #pragma unroll
-                    for (int j = 0; j < kChunk / 8; ++j) {
-                        // B operand: 8 K-columns of A^T = two core-matrix columns, 2048 bytes apart; 8-row groups 128 bytes apart
-                        const uint64_t bd = smem_desc(wbase + (uint32_t)(c * (kChunk / 4) + j * 2) * 2048u, 2048u, 128u);
-                        const uint32_t acc = (c > 0 || j > 0) ? 1u : 0u;
-                        mma_tf32_ts(tmem + kDhi, a_hi + j * 8, bd, acc);
-                        mma_tf32_ts(tmem + kDlo, a_lo + j * 8, bd, acc);
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t a_hi = tmem + kA0 + s * 64 + h * 32, a_lo = a_hi + 16;
+#pragma unroll
+                        for (int j = 0; j < kChunk / 8; ++j) {
+                            // B operand: 8 K-columns of A^T = two core-matrix columns, 2048 bytes apart; 8-row groups 128 bytes apart
+                            const uint64_t bd = smem_desc(wbase + (uint32_t)((c + h) * (kChunk / 4) + j * 2) * 2048u, 2048u, 128u);
+                            const uint32_t acc = (c > 0 || h > 0 || j > 0) ? 1u : 0u;
+                            mma_tf32_ts(tmem + kDhi, a_hi + j * 8, bd, acc);
+                            mma_tf32_ts(tmem + kDlo, a_lo + j * 8, bd, acc);
+                        }
                     }
                     mma_commit(&cb->a_empty[s]);
                 }
@@ -301,9 +308,9 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         if (!ok && lane == 0) { atomicCAS(err_word, 0, ERR_TC_WAIT | 5); cb->abort_flag = 1; }
     } else if (warp >= 4 && warp < 12) {
         // ------------------------------------------------ converters (lane quarter = warp % 4): two groups of four
-        // warps, the first takes the even chunks, the second the odd ones (a chunk's tensor-memory stage has the
-        // chunk's parity, kStages being even).  With one group the converter warps, at one busy warp per scheduler,
-        // ran at ~0.2 instructions per cycle and set the pace of the block (measured).
+        // warps, the first takes the even chunks, the second the odd ones; a tensor-memory stage holds one chunk of
+        // each (32 columns per group: hi 16 + lo 16).  With one group the converter warps, at one busy warp per
+        // scheduler, ran at ~0.2 instructions per cycle and set the pace of the block (measured).
         const int par = (warp - 4) >> 2;
         const int col = ((warp - 4) & 3) * 32 + lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -323,7 +330,7 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         int rs = par;              // raw stage of chunk q and its phase bit, advanced by hand (3 <= raw_stages <= 8)
         uint32_t rph = 0;
         for (int64_t q = par; q < total; q += 2) {
-            const int s = (int)(q & (kStages - 1));
+            const int s = (int)((q >> 1) & (kAStages - 1));
             // With an odd number of raw stages a stage alternates between the two groups, and this group may get here
             // before the other one has even seen the stage's previous chunk: the parity test on raw_full would then
             // pass on that older phase.  So first make sure the previous chunk of the stage has been released.
@@ -335,9 +342,9 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
 #pragma unroll
             for (int u = 0; u < kChunk; ++u) x[u] = r[u * kTile];
             if (pending >= 0) publish();
-            if (!mb_wait(&cb->a_empty[s], (uint32_t)(((q / kStages) & 1) ^ 1), abort_flag)) { ok = false; break; }
+            if (!mb_wait(&cb->a_empty[s], (uint32_t)((((q >> 1) / kAStages) & 1) ^ 1), abort_flag)) { ok = false; break; }
             fence_after();
-            uint32_t v[2 * kChunk];                      // hi in columns 0..15 of the stage, lo in 16..31
+            uint32_t v[2 * kChunk];                      // hi in columns 0..15 of this group's half of the stage, lo in 16..31
 #pragma unroll
             for (int u = 0; u < kChunk; ++u) {
                 v[u] = to_tf32(x[u]);
@@ -345,7 +352,7 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             }
             __syncwarp();
             if (lane == 0) mb_arrive(&cb->raw_empty[rs]);   // the raw chunk is in registers
-            tmem_st32(tmem + lane_base + kA0 + s * 32, v);
+            tmem_st32(tmem + lane_base + kA0 + s * 64 + par * 32, v);
             pending = s;
             rs += 2;
             if (rs >= raw_stages) { rs -= raw_stages; rph ^= 1u; }
