@@ -23,7 +23,7 @@
 //   warps 12-19 epilogue, two groups owning 64 workers each: tcgen05.ld both accumulators, add, release them, then
 //               y = acc/den - lr*g written over g in shared memory, quarter by quarter
 // Tensor memory (512 columns): D_hi 0..127, D_lo 128..255, four A stages of 64 columns (two chunks of hi 16 + lo 16).
-// Shared memory: control block, A^T (Kpad x 512 B), the G tile (64 KB), 3..8 raw stages of 8 KB.
+// Shared memory: control block, A^T (Kpad x 512 B), four (or two) 16 KB gradient / result quarters, 3..8 raw stages of 8 KB.
 // Every wait is bounded; a time-out sets the error word and lets the block run to its normal exit,
 // where tensor memory is released.
 #include <cuda.h>            // CUtensorMap and the cuTensorMapEncodeTiled prototype only; no libcuda link
@@ -44,7 +44,7 @@ constexpr int kAStages = 4;         // tensor-memory A stages of two chunks each
 constexpr int kThreads = 20 * 32;
 constexpr uint32_t kSpin = 1u << 20;
 constexpr int kRawStageBytes = kChunk * kTile * 4;          // 8 KB
-constexpr int kGTileBytes = 128 * kTile * 4;                // 64 KB
+constexpr int kGQuarterBytes = 32 * kTile * 4;              // 16 KB: 32 workers x 128 columns of gradients / results
 enum : int32_t { ERR_TC_WAIT = 3 << 24 };
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -165,13 +165,16 @@ __global__ void __launch_bounds__(kThreads, 1)
 mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapG,
                     const __grid_constant__ CUtensorMap mapY, int box_store,
                     float* __restrict__ X, int64_t P, int n_workers, float lr, const float* __restrict__ Wk,
-                    const HopTcRow* __restrict__ tbl, const int32_t* __restrict__ src_row, int Kpad, int raw_stages,
+                    const HopTcRow* __restrict__ tbl, const int32_t* __restrict__ src_row, int Kpad, int raw_stages, int g_bufs,
                     int32_t* __restrict__ err_word, const __grid_constant__ TcRowConsts rc) {
     extern __shared__ __align__(1024) unsigned char smem[];
     TcSmem* cb = reinterpret_cast<TcSmem*>(smem);
     float* Wsm = reinterpret_cast<float*>(smem + 4096);                        // Kpad * 512 bytes, canonical K-major
-    float* Gsm = reinterpret_cast<float*>(smem + 4096 + (size_t)Kpad * 512);   // [128 workers][128 columns]
-    float* raw = Gsm + 128 * kTile;                                            // raw_stages x [16][128] floats
+    // Gradient / result quarters of [32 workers][128 columns]: four buffers (one per quarter of the tile), or two (one per
+    // epilogue group, used for its two quarters in turn) when the weight matrix leaves too little room for raw stages
+    float* Gsm = reinterpret_cast<float*>(smem + 4096 + (size_t)Kpad * 512);
+    float* raw = Gsm + g_bufs * 32 * kTile;                                    // raw_stages x [16][128] floats
+    auto g_buf = [&](int q) -> float* { return Gsm + (g_bufs == 4 ? q : (q >> 1)) * 32 * kTile; };
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int64_t tiles = P / kTile;
     const int nchunks = Kpad / kChunk;
@@ -272,22 +275,26 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         auto refill = [&](int q, int64_t tile) {
             if (has_g) {
                 mb_expect_tx(&cb->g_full[q], qbytes);
-                tma_tile2d(Gsm + q * 32 * kTile, &mapG, (int)(tile * kTile), q * 32, &cb->g_full[q]);
+                tma_tile2d(g_buf(q), &mapG, (int)(tile * kTile), q * 32, &cb->g_full[q]);
             } else {
                 mb_arrive(&cb->g_full[q]);
             }
         };
+        // With two buffers a buffer serves quarters 2h and 2h+1 of a tile in turn: the even quarters go first, and
+        // what a buffer is refilled with after a store is the next quarter that lives in it.
+        const int n_even = (nq + 1) / 2;
         if (lane == 0 && (int64_t)blockIdx.x < tiles)
-            for (int q = 0; q < nq; ++q) refill(q, blockIdx.x);
+            for (int q = 0; q < nq; q += (g_bufs == 4 ? 1 : 2)) refill(q, blockIdx.x);
         int64_t tcount = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tcount) {
-            for (int q = 0; q < nq; ++q) {
+            for (int i = 0; i < nq; ++i) {
+                const int q = g_bufs == 4 ? i : (i < n_even ? 2 * i : 2 * (i - n_even) + 1);
                 if (!mb_wait(&cb->y_full[q], (uint32_t)(tcount & 1), abort_flag)) { ok = false; break; }
                 if (box_store) {
                     if (lane == 0) {   // all workers active: one box [32 workers x 128] into the output slot
                         asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-                                     ::"l"(&mapY), "r"((int)(tile * kTile)), "r"(q * 32), "r"(s32(Gsm + q * 32 * kTile)) : "memory");
+                                     ::"l"(&mapY), "r"((int)(tile * kTile)), "r"(q * 32), "r"(s32(g_buf(q))) : "memory");
                         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                     }
@@ -295,13 +302,18 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                     const HopTcRow rw = cb->rows[q * 32 + lane];
                     if (rw.out_row >= 0) {
                         asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                                     ::"l"(X + (int64_t)rw.out_row * P + tile * kTile), "r"(s32(Gsm + (q * 32 + lane) * kTile)), "r"(kTile * 4) : "memory");
+                                     ::"l"(X + (int64_t)rw.out_row * P + tile * kTile), "r"(s32(g_buf(q) + lane * kTile)), "r"(kTile * 4) : "memory");
                         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                     }
                 }
                 __syncwarp();          // the quarter has been read out of shared memory
-                if (lane == 0 && tile + gridDim.x < tiles) refill(q, tile + gridDim.x);
+                if (lane == 0) {
+                    const bool more = tile + gridDim.x < tiles;
+                    if (g_bufs == 4) { if (more) refill(q, tile + gridDim.x); }
+                    else if (!(q & 1) && q + 1 < nq) refill(q + 1, tile);
+                    else if (more) refill(q & ~1, tile + gridDim.x);
+                }
             }
         }
         asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // this thread's stores have reached global memory
@@ -392,7 +404,7 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                 if (q < nq && ok) {
                     if (!mb_wait(&cb->g_full[q], (uint32_t)(tcount & 1), abort_flag)) { ok = false; }
                     else {
-                        float* Gq = Gsm + q * 32 * kTile + col;
+                        float* Gq = g_buf(q) + col;
                         const float* dq = rc.inv_den + q * 32;
                         const uint32_t amq = rc.active_mask[q], gmq = rc.g_mask[q];
                         // Batches of 8 rows, the gradients of the next batch fetched before the stores of this one:
@@ -445,14 +457,19 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
 
 }  // namespace
 
-static int raw_stages_for(int Kpad) {
-    const long free_bytes = 227L * 1024 - 4096 - (long)Kpad * 512 - kGTileBytes;
-    return (int)std::max(0L, std::min<long>(kStages, free_bytes / kRawStageBytes));
+// Four gradient / result buffers when eight raw stages still fit beside them, else two (32 KB more for raw stages).
+static void tc_layout(int Kpad, int* g_bufs, int* raw_stages) {
+    const long free_bytes = 227L * 1024 - 4096 - (long)Kpad * 512;
+    const long st4 = std::min<long>(kStages, (free_bytes - 4 * kGQuarterBytes) / kRawStageBytes);
+    const long st2 = std::min<long>(kStages, (free_bytes - 2 * kGQuarterBytes) / kRawStageBytes);
+    *g_bufs = st4 >= kStages ? 4 : 2;
+    *raw_stages = (int)std::max(0L, *g_bufs == 4 ? st4 : st2);
 }
 // 0 when the level does not fit (fewer than 3 raw stages)
 size_t hop_dense_tc_smem(int Kpad) {
-    const int st = raw_stages_for(Kpad);
-    return st < 3 ? 0 : 4096 + (size_t)Kpad * 512 + kGTileBytes + (size_t)st * kRawStageBytes;
+    int gb, st;
+    tc_layout(Kpad, &gb, &st);
+    return st < 3 ? 0 : 4096 + (size_t)Kpad * 512 + (size_t)gb * kGQuarterBytes + (size_t)st * kRawStageBytes;
 }
 
 // Tensor maps: X as [N*(s+1) rows][P] with a one-row box of 128 columns (the tile::gather4 form loads four
@@ -520,11 +537,13 @@ int hop_launch_mix_dense_tc(const HopLaunchCfg& c, const void* mapX, const void*
         rc.g_mask[i >> 5] |= (uint32_t)(host_rows[i].g_row >= 0) << (i & 31);
     }
     const size_t smem = hop_dense_tc_smem(Kpad);
+    int gb, st;
+    tc_layout(Kpad, &gb, &st);
     cudaError_t e = hop_allow_max_smem<mix_dense_tc_kernel>();
     if (e != cudaSuccess) return (int)e;
     const int64_t tiles = c.P / kTile;
     const int grid = (int)std::min<int64_t>(tiles, (int64_t)c.sm_count);
     mix_dense_tc_kernel<<<grid, kThreads, smem, (cudaStream_t)c.stream>>>(mx, mg, my, mapY ? 1 : 0, c.X, c.P, c.N, c.lr, Wk, tbl, src_row, Kpad,
-                                                                          raw_stages_for(Kpad), c.err_word, rc);
+                                                                          st, gb, c.err_word, rc);
     return (int)cudaGetLastError();
 }
