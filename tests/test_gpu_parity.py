@@ -456,6 +456,26 @@ def test_tensor_path_with_a_ragged_last_quarter_of_workers():
     check(w, 1, TOL_STEP, hop.MIX_TENSOR, perturb=True)
 
 
+@pytest.mark.parametrize("N,s,b", [(40, 8, 4), (72, 3, 6)])
+def test_tensor_path_with_two_result_buffers(N, s, b):
+    # enough distinct consumed slices (K >= 192) that the weight matrix leaves room for only two of the four
+    # gradient / result buffers: each buffer then serves two quarters of the tile in turn.  N = 40: two quarters in one
+    # buffer, 9 ring slots so the rows leave by bulk copies; N = 72: three quarters, box stores.
+    P, iters = 128 * 6, 16
+    ptr, idx = inputs.graph_to_csr(inputs.complete(N))
+    rng = np.random.default_rng(31)
+    w = inputs.Workload(0, "dense-stale", N, P, iters, s=s, b=b, max_skip=0, max_ig=s, lr=0.05, momentum=0.0,
+                        weight_mode=inputs.STALE_LINEAR, grad_mode=inputs.GRAD_SYNTHETIC, in_ptr=ptr, in_idx=idx,
+                        ticks=rng.choice([1, 2, 9], size=(N, iters)).astype(np.uint64), grad_seed=5)
+    w._p0 = rng.standard_normal(P).astype(np.float32)
+    g = GpuRun(w, hop.MIX_TENSOR)
+    st = [g.h.level_stats(k) for k in range(iters)]
+    assert all(x["kernel"] == hop.MIX_TENSOR for x in st)
+    assert max(x["k_padded"] for x in st) >= 192
+    g.h.close()
+    check(w, iters, TOL_RUN, hop.MIX_TENSOR, perturb=True)
+
+
 def test_streaming_rejects_bad_records_and_run_checks_its_range():
     w = inputs.make_workload(4, P=256, iters=6)
     g = GpuRun(w)
