@@ -457,12 +457,14 @@ mix_dense_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
 
 }  // namespace
 
-// Four gradient / result buffers when eight raw stages still fit beside them, else two (32 KB more for raw stages).
+// Four gradient / result buffers while at least seven raw stages fit beside them, else two (32 KB more for raw
+// stages).  Two buffers put a load latency inside each epilogue group's chain, which costs ~10 % when the raw stages
+// were not the limit (K = 192, measured); with five or fewer raw stages the stages matter more (K >= 224).
 static void tc_layout(int Kpad, int* g_bufs, int* raw_stages) {
     const long free_bytes = 227L * 1024 - 4096 - (long)Kpad * 512;
     const long st4 = std::min<long>(kStages, (free_bytes - 4 * kGQuarterBytes) / kRawStageBytes);
     const long st2 = std::min<long>(kStages, (free_bytes - 2 * kGQuarterBytes) / kRawStageBytes);
-    *g_bufs = st4 >= kStages ? 4 : 2;
+    *g_bufs = st4 >= kStages - 1 ? 4 : 2;
     *raw_stages = (int)std::max(0L, *g_bufs == 4 ? st4 : st2);
 }
 // 0 when the level does not fit (fewer than 3 raw stages)

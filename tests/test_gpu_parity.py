@@ -456,9 +456,9 @@ def test_tensor_path_with_a_ragged_last_quarter_of_workers():
     check(w, 1, TOL_STEP, hop.MIX_TENSOR, perturb=True)
 
 
-@pytest.mark.parametrize("N,s,b", [(40, 8, 4), (72, 3, 6)])
+@pytest.mark.parametrize("N,s,b", [(40, 8, 4), (72, 4, 6)])
 def test_tensor_path_with_two_result_buffers(N, s, b):
-    # enough distinct consumed slices (K >= 192) that the weight matrix leaves room for only two of the four
+    # enough distinct consumed slices (K >= 224) that the weight matrix leaves room for only two of the four
     # gradient / result buffers: each buffer then serves two quarters of the tile in turn.  N = 40: two quarters in one
     # buffer, 9 ring slots so the rows leave by bulk copies; N = 72: three quarters, box stores.
     P, iters = 128 * 6, 16
@@ -471,7 +471,7 @@ def test_tensor_path_with_two_result_buffers(N, s, b):
     g = GpuRun(w, hop.MIX_TENSOR)
     st = [g.h.level_stats(k) for k in range(iters)]
     assert all(x["kernel"] == hop.MIX_TENSOR for x in st)
-    assert max(x["k_padded"] for x in st) >= 192
+    assert max(x["k_padded"] for x in st) >= 224
     g.h.close()
     check(w, iters, TOL_RUN, hop.MIX_TENSOR, perturb=True)
 
