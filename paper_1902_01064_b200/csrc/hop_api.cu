@@ -309,6 +309,7 @@ static int plan_level(hop_ctx* c, HopLevelHost& L, bool allow_tensor = true) {
             const int i = r.worker;
             L.tc_rows[i] = HopTcRow{r.out_row, (r.g_stage >= 0 && use_g) ? i : -1, 1.0f / (float)L.rec_den[a]};
             for (int t = r.ent_begin; t < r.ent_begin + r.ent_count; ++t) {
+                if (L.ent_num[t] == 0) continue;                 // padding entry
                 const int u = L.ent_slice[t];
                 // A^T in the K-major core-matrix layout the MMA reads: [u/4][i/8][i%8][u%4]
                 L.tc_w[(size_t)(u / 4) * 512 + (i / 8) * 32 + (i % 8) * 4 + (u % 4)] = (float)L.ent_num[t];

@@ -26,7 +26,7 @@ struct HopRecord {          // one active (NORMAL or JUMP) worker of a level
     int32_t self_u;         // float offset of the worker's own consumed slice inside a staged tile (weight decay)
     int32_t pad1;
 };
-struct HopEntry {
+struct alignas(8) HopEntry {
     int32_t u;              // float offset of the slice's row inside a staged tile: slice index * tile width
     float w;                // float(num) / float(den)
 };

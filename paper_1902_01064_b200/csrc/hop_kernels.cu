@@ -160,17 +160,78 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after kSpinLimit polls so that a lost copy can never hang the GPU.
+// Bounded wait: gives up after kSpinLimit polls so that a lost copy can never hang the GPU.  A failed poll is followed
+// by a sleep of SLEEP_NS: a poll returns after ~50 ns, and back-to-back polling by the waiting warps made up about
+// half of all instructions the kernel executed (ncu: 1150 polls per tile).
+template <int SLEEP_NS>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (it > 64) __nanosleep(64);
+        __nanosleep(SLEEP_NS);
     }
     return false;
 }
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+// A record as the bulk kernel keeps it in shared memory: everything that does not depend on the tile is worked out
+// once per block (the generic record costs ~60 instructions per tile and record in address arithmetic and flags).
+struct alignas(16) BulkRec {
+    int64_t out_off;        // out_row * P
+    int32_t ent_begin;      // first entry (a multiple of 4: entries are padded per record)
+    int32_t groups;         // entries / 4
+    int32_t g_off;          // float offset of the gradient row inside a staged tile, -1 without gradient
+    int32_t self_off;       // float offset of the worker's own consumed slice when weight decay applies, else -1
+    int32_t worker;
+    int32_t pad;
+};
+static_assert(sizeof(BulkRec) == sizeof(HopRecord), "the two record forms share the table space");
+
+// Reduce + Apply for one record and one tile from the shared-memory tables: whole groups of four entries, two
+// entries per 16-byte table load, the four slice loads of a group ahead of its multiply-adds (in entry order).
+template <bool MOMENTUM, bool DECAY>
+__device__ __forceinline__ void bulk_record(const BulkRec& r, const int4* __restrict__ ents2, const float* __restrict__ stage,
+                                            int w, int wd, int nG, float lr, float mu, float lam, float* __restrict__ Xc,
+                                            float* __restrict__ Mc, int64_t P, int lane) {
+    for (int c = lane * 4; c < wd; c += 128) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float* sc = stage + c;
+        const int4* e = ents2 + (r.ent_begin >> 1);
+#define HOP_FMA4(W, V) acc.x = fmaf(W, V.x, acc.x); acc.y = fmaf(W, V.y, acc.y); acc.z = fmaf(W, V.z, acc.z); acc.w = fmaf(W, V.w, acc.w)
+        for (int g = 0; g < r.groups; ++g, e += 2) {
+            const int4 e01 = e[0], e23 = e[1];             // (offset, weight) x 2 each
+            const float4 v0 = *reinterpret_cast<const float4*>(sc + e01.x);
+            const float4 v1 = *reinterpret_cast<const float4*>(sc + e01.z);
+            const float4 v2 = *reinterpret_cast<const float4*>(sc + e23.x);
+            const float4 v3 = *reinterpret_cast<const float4*>(sc + e23.z);
+            const float w0 = __int_as_float(e01.y), w1 = __int_as_float(e01.w), w2 = __int_as_float(e23.y), w3 = __int_as_float(e23.w);
+            HOP_FMA4(w0, v0); HOP_FMA4(w1, v1); HOP_FMA4(w2, v2); HOP_FMA4(w3, v3);
+        }
+#undef HOP_FMA4
+        if (DECAY && r.self_off >= 0 && r.g_off < 0) {
+            const float4 xs = *reinterpret_cast<const float4*>(sc + r.self_off);
+            const float k = -lr * lam;
+            acc.x = fmaf(k, xs.x, acc.x); acc.y = fmaf(k, xs.y, acc.y); acc.z = fmaf(k, xs.z, acc.z); acc.w = fmaf(k, xs.w, acc.w);
+        }
+        if (r.g_off >= 0) {
+            float4 g = *reinterpret_cast<const float4*>(sc + r.g_off);
+            if (DECAY && r.self_off >= 0) {
+                const float4 xs = *reinterpret_cast<const float4*>(sc + r.self_off);
+                g.x = fmaf(lam, xs.x, g.x); g.y = fmaf(lam, xs.y, g.y); g.z = fmaf(lam, xs.z, g.z); g.w = fmaf(lam, xs.w, g.w);
+            }
+            if constexpr (MOMENTUM) {
+                const float4 m = *reinterpret_cast<const float4*>(sc + r.g_off + nG * w);
+                g.x = fmaf(mu, m.x, g.x); g.y = fmaf(mu, m.y, g.y);
+                g.z = fmaf(mu, m.z, g.z); g.w = fmaf(mu, m.w, g.w);
+                *reinterpret_cast<float4*>(Mc + (int64_t)r.worker * P + c) = g;
+            }
+            acc.x = fmaf(-lr, g.x, acc.x); acc.y = fmaf(-lr, g.y, acc.y);
+            acc.z = fmaf(-lr, g.z, acc.z); acc.w = fmaf(-lr, g.w, acc.w);
+        }
+        *reinterpret_cast<float4*>(Xc + r.out_off + c) = acc;
+    }
 }
 
 // mix_bulk: persistent blocks; the first kProducerWarps warps are producers (asynchronous bulk copies of
@@ -186,16 +247,27 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw);
     uint64_t* empty = full + kBulkStages;
     float* stage0 = reinterpret_cast<float*>(smem_raw + 128 + table_bytes);
-    // the level's records and entries are read once per tile by every consumer warp: keep them on chip
-    const HopRecord* recs = lv.recs;
-    const HopEntry* ents = lv.ents;
+    // the level's records and entries are read once per tile by every consumer warp: keep them on chip, the records
+    // in the tile-independent form (when the tables do not fit, the consumers use the generic records in global memory)
+    BulkRec* srec = reinterpret_cast<BulkRec*>(smem_raw + 128);
+    const int4* sent2 = reinterpret_cast<const int4*>(srec + lv.nA);
     if (table_bytes > 0) {
-        HopRecord* srec = reinterpret_cast<HopRecord*>(smem_raw + 128);
-        HopEntry* sent = reinterpret_cast<HopEntry*>(srec + lv.nA);
-        const int4* gr = reinterpret_cast<const int4*>(lv.recs);
-        for (int i = threadIdx.x; i < lv.nA * 2; i += blockDim.x) reinterpret_cast<int4*>(srec)[i] = gr[i];
-        for (int i = threadIdx.x; i < n_ents; i += blockDim.x) sent[i] = lv.ents[i];
-        recs = srec; ents = sent;
+        for (int i = threadIdx.x; i < lv.nA; i += blockDim.x) {
+            const HopRecord r = lv.recs[i];
+            const bool grad = use_g != 0 && r.g_stage >= 0;
+            BulkRec b;
+            b.out_off = (int64_t)r.out_row * P;
+            b.ent_begin = r.ent_begin;
+            b.groups = r.ent_count >> 2;
+            b.g_off = grad ? (lv.U + r.g_stage) * w : -1;
+            b.self_off = (DECAY && r.g_stage >= 0 && r.self_u >= 0) ? r.self_u : -1;
+            b.worker = r.worker;
+            b.pad = 0;
+            srec[i] = b;
+        }
+        int2* sent = reinterpret_cast<int2*>(srec + lv.nA);
+        const int2* ge = reinterpret_cast<const int2*>(lv.ents);
+        for (int i = threadIdx.x; i < n_ents; i += blockDim.x) sent[i] = ge[i];
     }
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nG = use_g ? lv.nG : 0;
@@ -232,7 +304,7 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++n) {
             const int s = (int)(n % kBulkStages);
             const uint32_t ph = (uint32_t)((n / kBulkStages) & 1);
-            if (!mbar_wait(&empty[s], ph ^ 1u)) { ok = false; if (lane == 0) atomicCAS(err_word, 0, ERR_EMPTY_WAIT | (int)(tile & 0xffffff)); break; }
+            if (!mbar_wait<256>(&empty[s], ph ^ 1u)) { ok = false; if (lane == 0) atomicCAS(err_word, 0, ERR_EMPTY_WAIT | (int)(tile & 0xffffff)); break; }
             const int64_t c0 = tile * w;
             const int wd = (int)min((int64_t)w, P - c0);
             const uint32_t bytes = (uint32_t)wd * 4u;
@@ -249,7 +321,7 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
         if (ok) {
             const int64_t issued = n;
             for (int64_t m = (issued > kBulkStages ? issued - kBulkStages : 0); m < issued; ++m)
-                mbar_wait(&full[m % kBulkStages], (uint32_t)((m / kBulkStages) & 1));
+                mbar_wait<256>(&full[m % kBulkStages], (uint32_t)((m / kBulkStages) & 1));
         }
     } else {
         // ---------------- consumers
@@ -258,12 +330,17 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
         for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++n) {
             const int s = (int)(n % kBulkStages);
             const uint32_t ph = (uint32_t)((n / kBulkStages) & 1);
-            if (!mbar_wait(&full[s], ph)) { if (lane == 0) atomicCAS(err_word, 0, ERR_FULL_WAIT | (int)(tile & 0xffffff)); break; }
+            if (!mbar_wait<32>(&full[s], ph)) { if (lane == 0) atomicCAS(err_word, 0, ERR_FULL_WAIT | (int)(tile & 0xffffff)); break; }
             const int64_t c0 = tile * w;
             const int wd = (int)min((int64_t)w, P - c0);
             const float* st = stage0 + s * stage_floats;
-            for (int a = cw; a < lv.nA; a += kConsumerWarps)
-                reduce_apply_record<4, MOMENTUM, DECAY>(recs[a], ents, st, w, wd, lv.U, nG, use_g != 0, lr, mu, lam, X, M, P, c0, lane);
+            if (table_bytes > 0) {
+                for (int a = cw; a < lv.nA; a += kConsumerWarps)
+                    bulk_record<MOMENTUM, DECAY>(srec[a], sent2, st, w, wd, nG, lr, mu, lam, X + c0, MOMENTUM ? M + c0 : nullptr, P, lane);
+            } else {
+                for (int a = cw; a < lv.nA; a += kConsumerWarps)
+                    reduce_apply_record<4, MOMENTUM, DECAY>(lv.recs[a], lv.ents, st, w, wd, lv.U, nG, use_g != 0, lr, mu, lam, X, M, P, c0, lane);
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[s]);
         }

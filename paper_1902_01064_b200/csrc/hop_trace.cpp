@@ -140,6 +140,14 @@ void hop_build_level(const HopGraph& g, int32_t s, int32_t level, const int32_t*
         }
         out.rec_den.push_back(den[i]);
         out.sumC += r.ent_count;
+        // Entries are padded to a multiple of four per record with weight-0 terms on the record's first slice
+        // (adding 0 * x changes nothing), so that the mix kernels run whole groups of four without a remainder loop.
+        while (r.ent_count % 4 != 0 && r.ent_count > 0) {
+            out.ents.push_back({out.ents[r.ent_begin].u, 0.0f});
+            out.ent_slice.push_back(out.ent_slice[r.ent_begin]);
+            out.ent_num.push_back(0);
+            ++r.ent_count;
+        }
         out.recs.push_back(r);
     }
     out.nA = (int32_t)out.recs.size();
