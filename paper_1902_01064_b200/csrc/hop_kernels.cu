@@ -21,7 +21,9 @@ namespace {
 
 constexpr int kStagedThreads = 256;
 constexpr int kConsumerWarps = 16;
-constexpr int kProducerWarps = 6;   // a warp issues ~25-40 ns per small bulk copy: 1 / 2 / 4 / 6 warps gave 2.9 / 4.4 / 5.7 / 5.9 TB/s, 8 no more (measured)
+constexpr int kProducerWarps = 8;   // a warp issues ~25-40 ns per small bulk copy, so several issue in parallel.  Measured with
+                                    // 16 consumer warps: 4 / 6 / 8 producer warps 6.64 / 6.33 / 6.70 TB/s (and 12+6 6.64, 12+10 6.30,
+                                    // 14+10 6.65, 10+10 6.63): every split but the two with 22 warps in all is within 1.5 %
 constexpr int kBulkThreads = 32 * (kConsumerWarps + kProducerWarps);
 constexpr int kBulkStages = 2;
 constexpr uint32_t kSpinLimit = 1u << 22;
