@@ -388,30 +388,35 @@ __device__ __forceinline__ void box_muller(uint32_t ra, uint32_t rb, float sigma
 }
 
 // Four independent Philox blocks per thread (groups q, q + 256, q + 512, q + 768 of four columns): the ten rounds of one block are
-// a serial dependency chain; interleaved chains keep the issue slots busy (2.1 -> 1.7 ms per launch, measured).
+// a serial dependency chain; interleaved chains keep the issue slots busy (2.1 -> 1.7 ms per launch, measured).  A thread block
+// covers kGradChunks consecutive chunks of 1024 groups, so that the launch and drain of a block are spread over more work.
+constexpr int kGradChunks = 4;
 __global__ void __launch_bounds__(256)
 synth_grad_kernel(float* __restrict__ G, int64_t P, HopLevelDev lv, uint32_t k0, uint32_t k1, float sigma, int64_t col_offset) {
     const int worker = lv.grad_workers[blockIdx.y];
-    const int64_t q0 = (int64_t)blockIdx.x * 1024 + threadIdx.x;          // local group of 4 columns
     float* row = G + (int64_t)worker * P;
     const bool vec = (P & 3) == 0;
-    uint32_t o[4][4];
+    const uint64_t gq0 = (uint64_t)(col_offset / 4);
+#pragma unroll 1
+    for (int it = 0; it < kGradChunks; ++it) {
+        const int64_t q0 = ((int64_t)blockIdx.x * kGradChunks + it) * 1024 + threadIdx.x;   // local group of 4 columns
+        if (q0 * 4 >= P) break;
+        uint32_t o[4][4];
 #pragma unroll
-    for (int h = 0; h < 4; ++h) {
-        const uint64_t gq = (uint64_t)(col_offset / 4 + q0 + h * 256);
-        philox4x32_10((uint32_t)gq, (uint32_t)worker, (uint32_t)lv.level, 6u, k0, k1, o[h]);
-    }
+        for (int h = 0; h < 4; ++h)
+            philox4x32_10((uint32_t)(gq0 + q0 + h * 256), (uint32_t)worker, (uint32_t)lv.level, 6u, k0, k1, o[h]);
 #pragma unroll
-    for (int h = 0; h < 4; ++h) {
-        const int64_t c = (q0 + h * 256) * 4;
-        if (c >= P) continue;
-        float z[4];
-        box_muller(o[h][0], o[h][1], sigma, z[0], z[1]);
-        box_muller(o[h][2], o[h][3], sigma, z[2], z[3]);
-        if (vec) {
-            *reinterpret_cast<float4*>(row + c) = make_float4(z[0], z[1], z[2], z[3]);
-        } else {
-            for (int e = 0; e < 4 && c + e < P; ++e) row[c + e] = z[e];
+        for (int h = 0; h < 4; ++h) {
+            const int64_t c = (q0 + h * 256) * 4;
+            if (c >= P) continue;
+            float z[4];
+            box_muller(o[h][0], o[h][1], sigma, z[0], z[1]);
+            box_muller(o[h][2], o[h][3], sigma, z[2], z[3]);
+            if (vec) {
+                *reinterpret_cast<float4*>(row + c) = make_float4(z[0], z[1], z[2], z[3]);
+            } else {
+                for (int e = 0; e < 4 && c + e < P; ++e) row[c + e] = z[e];
+            }
         }
     }
 }
@@ -614,7 +619,7 @@ int hop_launch_mix_bulk(const HopLaunchCfg& c, const HopLevelDev& lv) {
 int hop_launch_synth_grad(const HopLaunchCfg& c, const HopLevelDev& lv, uint64_t seed, float sigma, int64_t col_offset) {
     if (lv.nG == 0) return 0;
     const int64_t groups = (c.P + 3) / 4;
-    dim3 grid((unsigned)((groups + 1023) / 1024), (unsigned)lv.nG);
+    dim3 grid((unsigned)((groups + 1024 * kGradChunks - 1) / (1024 * kGradChunks)), (unsigned)lv.nG);
     synth_grad_kernel<<<grid, 256, 0, (cudaStream_t)c.stream>>>(c.G, c.P, lv, (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), sigma, col_offset);
     return (int)cudaGetLastError();
 }
