@@ -129,6 +129,48 @@ def oracle_sample(w, budget_cols=131072, levels=6):
     return value, desc
 
 
+def _oracle_columns_task(job):
+    """Pool worker: the oracle's update rules on one chunk of the sampled columns (synthetic-gradient workloads
+    are separable by column).  A job without a trace only warms the process up (imports)."""
+    from oracle import update
+    if job is None:
+        return 0.0
+    tr, N, lr, momentum, p0, seed, sigma, cols, levels, s = job
+    t0 = time.perf_counter()
+    update.run_updates(tr, N, lr, momentum, np.tile(p0, (N, 1)), update.GradSynthetic(seed, sigma, cols), levels=levels, s=s)
+    return time.perf_counter() - t0
+
+
+def oracle_sample_all_cores(w, budget_cols=32768, levels=6):
+    """The same oracle sample with the sampled columns dealt to one process per available host core
+    (spawned, so that no child inherits a CUDA context).  Returns (value, cores) or None when the workload is not
+    separable by column (the SVM configurations) or only one core is available; `budget_cols` columns per process."""
+    import multiprocessing as mp
+    from oracle import protocol
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    cores = min(cores, 64)
+    if w.grad_mode != 1 or cores < 2:
+        return None
+    t0 = time.perf_counter()
+    tr = protocol.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode).to_arrays()
+    t_sim = time.perf_counter() - t0
+    levels = min(levels, w.iters)
+    C = min(w.P, budget_cols * cores)
+    cols = np.arange(C, dtype=np.int64) * (w.P // C)
+    p0 = w.p0()[cols].astype(np.float64)
+    chunks = np.array_split(np.arange(C), cores)
+    jobs = [(tr, w.N, w.lr, w.momentum, p0[c], w.grad_seed, w.sigma, cols[c], levels, w.s) for c in chunks]
+    with mp.get_context("spawn").Pool(cores) as pool:
+        pool.map(_oracle_columns_task, [None] * cores)          # processes up, modules imported
+        t0 = time.perf_counter()
+        pool.map(_oracle_columns_task, jobs, chunksize=1)
+        t_upd = time.perf_counter() - t0
+    n_wi = int((tr["op"][:levels] == 1).sum())
+    total_wi = int((tr["op"] == 1).sum())
+    per_wi = t_upd / n_wi * (w.P / C)
+    return total_wi / (t_sim + per_wi * total_wi), cores, C, t_upd
+
+
 def run_reference(args):
     """CPU oracle arm: same config, metric and unit; each step is a bounded sample."""
     rank = int(os.environ.get("RANK", "0"))
@@ -383,6 +425,15 @@ def main():
         wf = inputs.make_workload(args.config, P=args.P)
         v, desc = oracle_sample(wf)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
+        try:
+            allc = oracle_sample_all_cores(wf)
+        except Exception as ex:       # a baseline leg must never take the bench line down
+            allc = None
+            line["cpu_baseline"]["all_cores_error"] = repr(ex)
+        if allc is not None:
+            line["cpu_baseline"]["all_cores"] = {"value": allc[0], "unit": UNIT, "cores": allc[1],
+                                                 "sample": f"same update rules on {allc[2]} columns dealt to {allc[1]} processes "
+                                                           f"({allc[3]:.2f} s), protocol simulation serial"}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
