@@ -257,24 +257,6 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
     // in the tile-independent form (when the tables do not fit, the consumers use the generic records in global memory)
     BulkRec* srec = reinterpret_cast<BulkRec*>(smem_raw + 128);
     const int4* sent2 = reinterpret_cast<const int4*>(srec + lv.nA);
-    if (table_bytes > 0) {
-        for (int i = threadIdx.x; i < lv.nA; i += blockDim.x) {
-            const HopRecord r = lv.recs[i];
-            const bool grad = use_g != 0 && r.g_stage >= 0;
-            BulkRec b;
-            b.out_off = (int64_t)r.out_row * P;
-            b.ent_begin = r.ent_begin;
-            b.groups = r.ent_count >> 2;
-            b.g_off = grad ? (lv.U + r.g_stage) * w : -1;
-            b.self_off = (DECAY && r.g_stage >= 0 && r.self_u >= 0) ? r.self_u : -1;
-            b.worker = r.worker;
-            b.pad = 0;
-            srec[i] = b;
-        }
-        int2* sent = reinterpret_cast<int2*>(srec + lv.nA);
-        const int2* ge = reinterpret_cast<const int2*>(lv.ents);
-        for (int i = threadIdx.x; i < n_ents; i += blockDim.x) sent[i] = ge[i];
-    }
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nG = use_g ? lv.nG : 0;
     const int rows = lv.U + nG * (MOMENTUM ? 2 : 1);
@@ -332,6 +314,29 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
     } else {
         // ---------------- consumers
         const int cw = warp - kProducerWarps;
+        // The tables are built by the consumer warps alone, behind a barrier of their own, while the producers are
+        // already fetching the first tiles.
+        if (table_bytes > 0) {
+            constexpr int kConsumerThreads = 32 * kConsumerWarps;
+            const int ct = tid - 32 * kProducerWarps;
+            for (int i = ct; i < lv.nA; i += kConsumerThreads) {
+                const HopRecord r = lv.recs[i];
+                const bool grad = use_g != 0 && r.g_stage >= 0;
+                BulkRec b;
+                b.out_off = (int64_t)r.out_row * P;
+                b.ent_begin = r.ent_begin;
+                b.groups = r.ent_count >> 2;
+                b.g_off = grad ? (lv.U + r.g_stage) * w : -1;
+                b.self_off = (DECAY && r.g_stage >= 0 && r.self_u >= 0) ? r.self_u : -1;
+                b.worker = r.worker;
+                b.pad = 0;
+                srec[i] = b;
+            }
+            int2* sent = reinterpret_cast<int2*>(srec + lv.nA);
+            const int2* ge = reinterpret_cast<const int2*>(lv.ents);
+            for (int i = ct; i < n_ents; i += kConsumerThreads) sent[i] = ge[i];
+            asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
+        }
         int64_t n = 0;
         for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++n) {
             const int s = (int)(n % kBulkStages);
