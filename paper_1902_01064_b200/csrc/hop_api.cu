@@ -159,6 +159,7 @@ extern "C" int hop_destroy(hop_ctx* c) {
 
 extern "C" int hop_set_option(hop_ctx* c, int key, double v) {
     if (!c) return HOP_E_ARG;
+    if (!std::isfinite(v)) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: the value must be finite");
     drop_graphs(c);
     if (key == HOP_OPT_USE_GRAPH) { c->use_graph = v != 0.0; return HOP_OK; }
     if (key == HOP_OPT_NOTIFY_ACK) { c->sp.notify_ack = v != 0.0; return HOP_OK; }
@@ -184,7 +185,7 @@ extern "C" int hop_set_option(hop_ctx* c, int key, double v) {
     }
     if (key >= HOP_OPT_BACKUP_OF_WORKER) {
         const int i = key - HOP_OPT_BACKUP_OF_WORKER;
-        if (i >= c->g.N) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: worker index out of range");
+        if (i < 0 || i >= c->g.N) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: worker index out of range");
         const int d = c->g.in_ptr[i + 1] - c->g.in_ptr[i];
         if (v < 0 || v >= d || v != std::floor(v)) HOP_FAIL(c, HOP_E_GRAPH, "hop_set_option: N_buw(i) must be an integer in [0, |N_in(i)|)");
         c->sp.b[i] = (int32_t)v;

@@ -48,7 +48,8 @@ def test_options_are_validated():
     ptr, idx = inputs.graph_to_csr(inputs.ring(4))
     h = hop.Hop(ptr, idx, 4, 16, 1, 0, 0)
     for key, val in [(hop.OPT_MAX_IG, -1), (hop.OPT_WEIGHT_MODE, 7), (hop.OPT_GRAD_MODE, 9), (hop.OPT_COL_OFFSET, 6),
-                     (hop.OPT_BACKUP_OF_WORKER + 1, 3), (hop.OPT_BACKUP_OF_WORKER + 9, 0), (77, 1)]:
+                     (hop.OPT_BACKUP_OF_WORKER + 1, 3), (hop.OPT_BACKUP_OF_WORKER + 9, 0), (77, 1),
+                     (hop.OPT_LR, float("nan")), (hop.OPT_GRAD_SIGMA, float("inf"))]:
         with pytest.raises(hop.HopError):
             h.set_option(key, val)
     h.set_option(hop.OPT_BACKUP_OF_WORKER + 2, 2)
