@@ -19,7 +19,7 @@
 
 namespace {
 
-constexpr int kStagedThreads = 256;
+constexpr int kStagedThreads = 512;
 constexpr int kConsumerWarps = 16;
 constexpr int kProducerWarps = 8;   // a warp issues ~25-40 ns per small bulk copy, so several issue in parallel.  Measured with
                                     // 16 consumer warps: 4 / 6 / 8 producer warps 6.64 / 6.33 / 6.70 TB/s (and 12+6 6.64, 12+10 6.30,
@@ -33,7 +33,9 @@ enum : int32_t { ERR_FULL_WAIT = 1 << 24, ERR_EMPTY_WAIT = 2 << 24 };
 // ------------------------------------------------------------------------------------------------
 // Consumer math shared by both mix kernels: one warp produces the tile of one record.
 // stage: [rows][w] floats; rows [0,U) consumed slices, [U,U+nG) gradients, [U+nG,U+2nG) momentum.
-template <int VEC, bool MOMENTUM, bool DECAY>
+// ALIGNED = false (VEC = 4 only): the rows of X and M are not 16-byte aligned in global memory (P % 4 != 0), so the
+// results leave as guarded scalar stores; shared memory is aligned either way.
+template <int VEC, bool MOMENTUM, bool DECAY, bool ALIGNED = true>
 __device__ __forceinline__ void reduce_apply_record(const HopRecord& r, const HopEntry* __restrict__ ents,
                                                     const float* __restrict__ stage, int w, int wd, int U, int nG,
                                                     bool use_g, float lr, float mu, float lam, float* __restrict__ X,
@@ -83,12 +85,24 @@ __device__ __forceinline__ void reduce_apply_record(const HopRecord& r, const Ho
                     const float4 m = *reinterpret_cast<const float4*>(mrow + c);
                     g.x = fmaf(mu, m.x, g.x); g.y = fmaf(mu, m.y, g.y);
                     g.z = fmaf(mu, m.z, g.z); g.w = fmaf(mu, m.w, g.w);
-                    *reinterpret_cast<float4*>(mout + c) = g;
+                    if constexpr (ALIGNED) {
+                        *reinterpret_cast<float4*>(mout + c) = g;
+                    } else {
+                        const float gv[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) if (c + q < wd) mout[c + q] = gv[q];
+                    }
                 }
                 acc.x = fmaf(-lr, g.x, acc.x); acc.y = fmaf(-lr, g.y, acc.y);
                 acc.z = fmaf(-lr, g.z, acc.z); acc.w = fmaf(-lr, g.w, acc.w);
             }
-            *reinterpret_cast<float4*>(out + c) = acc;
+            if constexpr (ALIGNED) {
+                *reinterpret_cast<float4*>(out + c) = acc;
+            } else {
+                const float av[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) if (c + q < wd) out[c + q] = av[q];
+            }
         } else {
             float acc = 0.f;
             for (int t = 0; t < n; ++t) {
@@ -111,37 +125,69 @@ __device__ __forceinline__ void reduce_apply_record(const HopRecord& r, const Ho
 }
 
 // ------------------------------------------------------------------------------------------------
-// mix_staged: ordinary loads into shared memory, one barrier, compute, one barrier.  Works for any P
-// (VEC = 1 when P is not a multiple of 4).
-template <int VEC, bool MOMENTUM, bool DECAY>
-__global__ void __launch_bounds__(kStagedThreads)
+// mix_staged: the general kernel, for any P.  Persistent blocks, two shared-memory stages filled with cp.async by all
+// threads (one warp per staged row), block-wide barriers: the copies of the next tile are in flight while this tile
+// is computed.  MODE 0: P % 4 == 0, 16-byte copies, vector math and stores.  MODE 1: any P with a tile width that is
+// a multiple of 4: 4-byte copies (the rows are not 16-byte aligned in global memory, the staged copy is), vector
+// math, scalar stores.  MODE 2: scalar everything (tile widths below 32 that are not multiples of 4).
+__device__ __forceinline__ void cp_async_4(float* dst, const float* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_16(float* dst, const float* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+template <int MODE, bool MOMENTUM, bool DECAY>
+__global__ void __launch_bounds__(kStagedThreads, 1)
 mix_staged_kernel(float* __restrict__ X, float* __restrict__ M, const float* __restrict__ G, int64_t P, int w,
                   int use_g, float lr, float mu, float lam, HopLevelDev lv) {
     extern __shared__ __align__(16) float smem[];
+    constexpr int kWarps = kStagedThreads / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nG = use_g ? lv.nG : 0;
+    const int rows = lv.U + nG * (MOMENTUM ? 2 : 1);
+    const int64_t stage_floats = (int64_t)rows * w;
     const int64_t tiles = (P + w - 1) / w;
-    for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    auto fetch = [&](int64_t tile, int stage) {
         const int64_t c0 = tile * w;
         const int wd = (int)min((int64_t)w, P - c0);
-        const int per_row = (wd + VEC - 1) / VEC;
-        const int rows = lv.U + nG * (MOMENTUM ? 2 : 1);
-        for (int idx = tid; idx < rows * per_row; idx += kStagedThreads) {
-            const int r = idx / per_row, c = (idx - r * per_row) * VEC;
+        float* dst0 = smem + stage * stage_floats;
+        for (int r = warp; r < rows; r += kWarps) {
             const float* src;
             if (r < lv.U) src = X + (int64_t)lv.src_row[r] * P;
             else if (r < lv.U + nG) src = G + (int64_t)lv.grad_workers[r - lv.U] * P;
             else src = M + (int64_t)lv.grad_workers[r - lv.U - nG] * P;
-            if constexpr (VEC == 4)
-                *reinterpret_cast<float4*>(smem + (int64_t)r * w + c) = *reinterpret_cast<const float4*>(src + c0 + c);
-            else
-                smem[(int64_t)r * w + c] = src[c0 + c];
+            src += c0;
+            float* dst = dst0 + (int64_t)r * w;
+            if constexpr (MODE == 0) {
+                for (int c = lane * 4; c < wd; c += 128) cp_async_16(dst + c, src + c);
+            } else {
+                for (int c = lane; c < wd; c += 32) cp_async_4(dst + c, src + c);
+            }
         }
-        __syncthreads();
-        for (int a = warp; a < lv.nA; a += kStagedThreads / 32)
-            reduce_apply_record<VEC, MOMENTUM, DECAY>(lv.recs[a], lv.ents, smem, w, wd, lv.U, nG, use_g != 0, lr, mu, lam, X, M, P, c0, lane);
-        __syncthreads();
+    };
+    int n = 0;
+    if ((int64_t)blockIdx.x < tiles) fetch(blockIdx.x, 0);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++n) {
+        const int64_t next = tile + gridDim.x;
+        if (next < tiles) fetch(next, (n + 1) & 1);
+        asm volatile("cp.async.commit_group;" ::: "memory");          // one group per iteration, empty or not
+        asm volatile("cp.async.wait_group 1;" ::: "memory");          // this tile's copies (of this thread) have landed
+        __syncthreads();                                               // ... and everybody else's
+        const int64_t c0 = tile * w;
+        const int wd = (int)min((int64_t)w, P - c0);
+        const float* st = smem + (n & 1) * stage_floats;
+        for (int a = warp; a < lv.nA; a += kWarps) {
+            if constexpr (MODE == 0)
+                reduce_apply_record<4, MOMENTUM, DECAY, true>(lv.recs[a], lv.ents, st, w, wd, lv.U, nG, use_g != 0, lr, mu, lam, X, M, P, c0, lane);
+            else if constexpr (MODE == 1)
+                reduce_apply_record<4, MOMENTUM, DECAY, false>(lv.recs[a], lv.ents, st, w, wd, lv.U, nG, use_g != 0, lr, mu, lam, X, M, P, c0, lane);
+            else
+                reduce_apply_record<1, MOMENTUM, DECAY>(lv.recs[a], lv.ents, st, w, wd, lv.U, nG, use_g != 0, lr, mu, lam, X, M, P, c0, lane);
+        }
+        __syncthreads();                                               // the stage may be refilled by the next iteration
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -556,25 +602,25 @@ apply_dense_kernel(float* __restrict__ X, float* __restrict__ M, const float* __
     }
 }
 
+constexpr int kStagedStages = 2;
 size_t staged_smem(const HopLaunchCfg& c, const HopLevelDev& lv) {
     const int nG = c.use_g ? lv.nG : 0;
     const int rows = lv.U + nG * (c.mu != 0.f ? 2 : 1);
-    return (size_t)rows * c.tile_w * sizeof(float);
+    return (size_t)kStagedStages * rows * c.tile_w * sizeof(float);
 }
 
 }  // namespace
 
-int hop_mix_smem_budget(int kernel) { return kernel == HOP_MIX_BULK ? (227 * 1024 - 128) : 100 * 1024; }
+int hop_mix_smem_budget(int kernel) { return kernel == HOP_MIX_BULK ? (227 * 1024 - 128) : 200 * 1024; }
 int hop_mix_table_limit() { return 32 * 1024; }
-int hop_mix_stages(int kernel) { return kernel == HOP_MIX_BULK ? kBulkStages : 1; }
+int hop_mix_stages(int kernel) { return kernel == HOP_MIX_BULK ? kBulkStages : kStagedStages; }
 
 int hop_launch_mix_staged(const HopLaunchCfg& c, const HopLevelDev& lv) {
     if (lv.nA == 0) return 0;
     const size_t smem = staged_smem(c, lv);
     const int64_t tiles = (c.P + c.tile_w - 1) / c.tile_w;
-    const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(8, (200 * 1024) / std::max<size_t>(smem, 1)));
-    const int grid = (int)std::min<int64_t>(tiles, (int64_t)c.sm_count * per_sm);
-    const bool vec = (c.P % 4 == 0) && (c.tile_w % 4 == 0);
+    const int grid = (int)std::min<int64_t>(tiles, (int64_t)c.sm_count);
+    const int mode = (c.P % 4 == 0 && c.tile_w % 4 == 0) ? 0 : (c.tile_w % 4 == 0 ? 1 : 2);
     const bool mom = c.mu != 0.f;
     cudaStream_t st = (cudaStream_t)c.stream;
     cudaError_t e = cudaSuccess;
@@ -585,10 +631,11 @@ int hop_launch_mix_staged(const HopLaunchCfg& c, const HopLevelDev& lv) {
             mix_staged_kernel<V, MO, DE><<<grid, kStagedThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, c.wd, lv); \
     } while (0)
 #define HOP_LAUNCH_STAGED2(V, MO) do { if (c.wd != 0.f) HOP_LAUNCH_STAGED(V, MO, true); else HOP_LAUNCH_STAGED(V, MO, false); } while (0)
-    if (vec && mom) HOP_LAUNCH_STAGED2(4, true);
-    else if (vec) HOP_LAUNCH_STAGED2(4, false);
-    else if (mom) HOP_LAUNCH_STAGED2(1, true);
-    else HOP_LAUNCH_STAGED2(1, false);
+#define HOP_LAUNCH_STAGED3(V) do { if (mom) HOP_LAUNCH_STAGED2(V, true); else HOP_LAUNCH_STAGED2(V, false); } while (0)
+    if (mode == 0) HOP_LAUNCH_STAGED3(0);
+    else if (mode == 1) HOP_LAUNCH_STAGED3(1);
+    else HOP_LAUNCH_STAGED3(2);
+#undef HOP_LAUNCH_STAGED3
 #undef HOP_LAUNCH_STAGED2
 #undef HOP_LAUNCH_STAGED
     if (e != cudaSuccess) return (int)e;
