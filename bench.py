@@ -33,7 +33,7 @@ PROBE = 1024
 # from the ncu captures summarised under profiles/: taken at a smaller parameter count and scaled by the number of
 # columns (traffic is proportional to columns at a fixed trace).  Dropped to None whenever the kernel changes.
 NCU_TRAFFIC = {(4, 25_600_000): 23.49e9,      # profiles/mix_bulk_kernel_cfg4.md, section 2b (all 50 levels, current kernel)
-               (5, 8_000_000): 12.65e9}       # profiles/mix_dense_tc_kernel_cfg5.md, section 2b (all 30 levels, current kernel)
+               (5, 8_000_000): 12.64e9}       # profiles/mix_dense_tc_kernel_cfg5.md, section 2b (all 30 levels, current kernel)
 
 
 def shard_columns(P: int, n: int, r: int, unit: int = 128):
