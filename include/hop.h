@@ -93,8 +93,9 @@ typedef enum hop_grad_mode {
 
 typedef enum hop_mix_kernel {
     HOP_MIX_AUTO = 0,
-    HOP_MIX_STAGED = 1,      /* column tile staged in shared memory with ordinary vector loads     */
-    HOP_MIX_BULK = 2,        /* same, slices fetched by asynchronous bulk copies in a pipeline     */
+    HOP_MIX_STAGED = 1,      /* column tile staged in shared memory by cp.async, two stages; any P */
+    HOP_MIX_BULK = 2,        /* same, slices fetched by bulk copies, producer and consumer warps;  */
+                             /* needs P % 4 == 0 (AUTO picks it then, else STAGED)                 */
     HOP_MIX_TENSOR = 3       /* dense graphs: W_k * X on tcgen05 tensor cores, 3xTF32              */
 } hop_mix_kernel;
 
