@@ -551,7 +551,15 @@ svm_dense_grad_kernel(float* __restrict__ G, int64_t P, HopLevelDev lv, const fl
     const float* a0 = A + ((int64_t)worker * R + (int64_t)(lv.level % (R / B)) * B) * P + p;
     const float* cf = coef + (int64_t)worker * B;
     float g = 0.f;
-    for (int r = 0; r < B; ++r) g = fmaf(cf[r], a0[(int64_t)r * P], g);
+    int r = 0;
+    for (; r + 8 <= B; r += 8) {          // eight independent loads in flight, the multiply-adds in row order
+        float a[8], c[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { a[i] = a0[(int64_t)(r + i) * P]; c[i] = cf[r + i]; }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) g = fmaf(c[i], a[i], g);
+    }
+    for (; r < B; ++r) g = fmaf(cf[r], a0[(int64_t)r * P], g);
     G[(int64_t)worker * P + p] = g;
 }
 
