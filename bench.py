@@ -103,7 +103,8 @@ def oracle_sample(w, budget_cols=131072, levels=6):
     to the full parameter count, description)."""
     from oracle import protocol, update
     t0 = time.perf_counter()
-    tr = protocol.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode).to_arrays()
+    tr = protocol.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode,
+                           stale_reduce=w.stale_reduce).to_arrays()
     t_sim = time.perf_counter() - t0
     levels = min(levels, w.iters)
     if w.grad_mode == 1:
@@ -152,7 +153,8 @@ def oracle_sample_all_cores(w, budget_cols=32768, levels=6):
     if w.grad_mode != 1 or cores < 2:
         return None
     t0 = time.perf_counter()
-    tr = protocol.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode).to_arrays()
+    tr = protocol.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode,
+                           stale_reduce=w.stale_reduce).to_arrays()
     t_sim = time.perf_counter() - t0
     levels = min(levels, w.iters)
     C = min(w.P, budget_cols * cores)

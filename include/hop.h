@@ -67,8 +67,19 @@ typedef enum hop_op {
  * STALE_LINEAR: numerator Iter(u) - (k - s) + 1, normalised (Eq. 2). */
 typedef enum hop_weight_mode { HOP_W_UNIFORM = 0, HOP_W_STALE_LINEAR = 1 } hop_weight_mode;
 
+/* Which usable updates enter the Reduce under bounded staleness (s > 0).  An in-neighbour is usable at
+ * iteration k when the newest update ever dequeued from it has iteration >= k - s; that decides blocking
+ * in both modes (Section 4.4: an older update still inside the bound needs no new arrival).
+ * NEW_ONLY (default, the printed rule): only updates this Recv itself dequeued are reduced -- Eq. 2 sums over
+ * the in-neighbours whose update received in iteration k is usable, and Fig. alg3's Recv appends an update
+ * only when the newest iteration among what the call dequeued is inside the bound.  A neighbour that has not
+ * advanced since the worker's previous Recv adds no term; the own update is always new.
+ * REUSE: such a neighbour's last update is reduced again with the smaller weight Eq. 2 gives its age, so every
+ * usable in-neighbour contributes at every iteration.  With s = 0 both coincide. */
+typedef enum hop_stale_reduce { HOP_STALE_NEW_ONLY = 0, HOP_STALE_REUSE = 1 } hop_stale_reduce;
+
 /* What Recv keeps once |N_in(i)| - N_buw(i) in-neighbours are usable.  AT_LEAST: every usable update
- * (Fig. alg4: the needed ones, then "any additional update" in the queue).  EXACT: exactly
+ * (Fig. alg4: the needed ones, then whatever else is queued for that iteration).  EXACT: exactly
  * |N_in(i)| - N_buw(i): the own update plus the neighbours whose first usable update was sent
  * earliest (what a FIFO dequeue of that many entries returns), ties by worker id. */
 typedef enum hop_backup_mode { HOP_BACKUP_AT_LEAST = 0, HOP_BACKUP_EXACT = 1 } hop_backup_mode;
@@ -119,6 +130,7 @@ typedef enum hop_option {
     HOP_OPT_WEIGHT_DECAY = 13,/* lambda >= 0: lambda * x_{k,i} is added to the gradient (Section 7.2 uses 1e-4 / 1e-7)  */
     HOP_OPT_LOSS = 14,        /* hop_loss of the SVM modes (default HINGE; the paper's runs used LOG, Section 7.2)    */
     HOP_OPT_APPROACH = 15,    /* hop_approach (default PARALLEL, the paper's choice, Section 3.2)                     */
+    HOP_OPT_STALE_REDUCE = 16,/* hop_stale_reduce (default NEW_ONLY: Eq. 2 / Fig. alg3 as printed)                    */
     HOP_OPT_BACKUP_OF_WORKER = 1000 /* key = 1000 + i sets N_buw(i) of one worker (Fig. alg4)       */
 } hop_option;
 
@@ -170,8 +182,10 @@ int hop_bind_svm_csr(hop_ctx* ctx, const int64_t* row_ptr, const int32_t* col, c
                      const float* y, int32_t rows_per_worker, int32_t batch);
 
 /* Validates every record on the host -- consumed neighbour in N_in(i), version in [k-s, k] and
- * actually produced, own update present, at least |N_in(i)| - b entries, positive numerators
- * summing to den, JUMP/IDLE consistent with the versions a worker holds -- then uploads the
+ * actually produced, own update present, at least |N_in(i)| - b entries (with s > 0 under
+ * HOP_STALE_NEW_ONLY: at least the own update), versions consumed over an edge never going back
+ * (and never repeating under HOP_STALE_NEW_ONLY), positive numerators summing to den,
+ * JUMP/IDLE consistent with the versions a worker holds -- then uploads the
  * per-level tables (cudaMalloc + H2D on the bound stream) and rewinds to level 0. */
 int hop_load_trace(hop_ctx* ctx, const hop_trace* t);
 

@@ -16,11 +16,21 @@ Readings taken where the paper is silent (listed once more in the design notes):
       iter <= k (Section 6: one queue per iteration slot keeps newer iterations out of
       reach); it is satisfactory iff iter >= k - s.  The newest update seen so far from j
       is remembered (Fig. alg3 iter_rcv; Section 4.4: an earlier update still inside the bound
-      needs no new arrival).
+      needs no new arrival, so it never blocks the worker).
+  R2' Which satisfactory updates enter the Reduce (stale_reduce).  NEW_ONLY, the default, is what
+      the paper prints three times: Eq. 2 sums over the in-neighbours whose update received in
+      iteration k is satisfactory, Fig. alg3's Recv appends an update only when the newest
+      iteration among what this call dequeued is inside the bound, and Section 4.4 reduces the
+      newly received updates.  An in-neighbour whose newest update was already taken out of the
+      queue by an earlier Recv of this worker still counts for the blocking test but adds no
+      term; the own update is new in every iteration.  REUSE adds such an update again, with the
+      lower weight Eq. 2 gives its age (every satisfactory in-neighbour contributes at every
+      level).
   R3  Recv(k, i) completes at the first moment at least |N_in(i)| - b_i in-neighbours (self
-      included) are satisfactory, and then consumes every satisfactory one (Fig. alg4: the
-      required number, then whatever else is there).  b = 0 is Fig. alg3, s = 0 is Fig. alg4,
-      both 0 is Fig. alg1; both > 0 is the "hybrid" row of Table 1.
+      included) are satisfactory, and then takes every satisfactory one (Fig. alg4: the
+      required number, then whatever else is there), subject to R2'.  b = 0 is Fig. alg3, s = 0 is
+      Fig. alg4 (an update of iteration k is first dequeued by Recv(k), so R2' changes nothing
+      there), both 0 is Fig. alg1; both > 0 is the "hybrid" row of Table 1.
   R4  Same-tick ordering: rounds.  In a round every worker decides its transition from the
       state left by the previous round; then all decisions are committed in worker order.
       One transition per worker per round; rounds repeat until nothing moves.
@@ -38,10 +48,11 @@ Readings taken where the paper is silent (listed once more in the design notes):
       the paper states for it (Table 1: a receiver at most 1 ahead of its sender, a sender at most 2 ahead of its
       receiver) and the Section 3.4 example (B and C stuck in iteration 1 waiting for ACK(0)); the Section 3.5
       remark that they could not even enter iteration 1 is at odds with both and is not followed.
-  R7  backup_exact (off by default; the paper's Fig. alg4 takes "any additional update"): Recv completes at the
+  R7  backup_exact (off by default; Fig. alg4 takes the required number, then whatever else is queued): Recv completes at the
       same moment as under R3 but keeps exactly |N_in(i)| - b_i updates: its own, plus those in-neighbours
       whose first satisfactory update (iter in [k-s, k]) arrived earliest in UpdateQ(i) (FIFO order of
       Fig. alg4's dequeue); the version taken from a kept neighbour is still its newest one with iter <= k.
+      Under NEW_ONLY the kept set is chosen first and R2' then drops the kept ones that are not new.
 """
 from __future__ import annotations
 
@@ -51,6 +62,7 @@ import numpy as np
 
 IDLE, NORMAL, JUMP = 0, 1, 2
 UNIFORM, STALE_LINEAR = 0, 1
+NEW_ONLY, REUSE = 0, 1
 
 _COMPUTE, _RECV, _TOKEN, _JUMPRECV, _DONE = range(5)
 
@@ -99,7 +111,8 @@ def reduce_weights(vers, level, s, weight_mode):
 
 class HopProtocol:
     def __init__(self, n_in, ticks, iters, s=0, b=0, max_ig=None, max_skip=0,
-                 weight_mode=UNIFORM, on_round=None, backup_exact=False, notify_ack=False):
+                 weight_mode=UNIFORM, on_round=None, backup_exact=False, notify_ack=False,
+                 stale_reduce=NEW_ONLY):
         self.N = N = len(n_in)
         self.n_in = [list(nb) for nb in n_in]
         for i, nb in enumerate(self.n_in):
@@ -132,6 +145,9 @@ class HopProtocol:
         self.arrival_pos = {}                                  # (w_id, i) -> {iter: position in UpdateQ(i)'s arrival order}
         self.update_q = [[] for _ in range(N)]                 # FIFO of (iter, w_id) tags
         self.iter_rcv = {(j, i): -1 for i in range(N) for j in self.n_in[i]}
+        self.stale_reduce = stale_reduce
+        # iter_rcv as it stood when worker i last completed a Recv: what that call (or an earlier one) dequeued
+        self.iter_reduced = {(j, i): -1 for i in range(N) for j in self.n_in[i]}
         self.token_q = {}
         if max_ig is not None:
             for i in range(N):
@@ -191,7 +207,15 @@ class HopProtocol:
             others = sorted((jv for jv in got if jv[0] != i), key=lambda jv: (first_satisfactory_arrival(jv[0]), jv[0]))
             keep = {i} | {j for j, _ in others[:need - 1]}
             got = [jv for jv in got if jv[0] in keep]
+        if self.stale_reduce == NEW_ONLY:
+            # Fig. alg3: only what this Recv call itself dequeued is appended (max(l_iter) >= min_iter)
+            got = [(j, v) for (j, v) in got if j == i or v > self.iter_reduced[(j, i)]]
         return got
+
+    def _recv_done(self, i):
+        """Recv of worker i returned: everything it dequeued, used or not, is gone from the queue."""
+        for j in self.n_in[i]:
+            self.iter_reduced[(j, i)] = self.iter_rcv[(j, i)]
 
     def _record(self, op, level, i, got, own_as=None):
         vers = [(own_as if (j == i and own_as is not None) else v) for (j, v) in got]
@@ -245,6 +269,7 @@ class HopProtocol:
         k = self.Iter[i]
         if act[0] == "applied":
             self._record(NORMAL, k, i, act[1])
+            self._recv_done(i)
             if self.notify_ack:
                 for j in self.n_in[i]:
                     if j != i:
@@ -259,6 +284,7 @@ class HopProtocol:
         elif act[0] == "jump":
             target, got = act[1], act[2]
             self._record(JUMP, target - 1, i, got, own_as=target - 1)
+            self._recv_done(i)
             self._take_tokens(i, target - k)
             self._enter(i, target, n_tokens=target - k)
 
@@ -289,8 +315,9 @@ class HopProtocol:
 
 
 def simulate(n_in, ticks, iters, s=0, b=0, max_ig=None, max_skip=0, weight_mode=UNIFORM, on_round=None,
-             backup_exact=False, notify_ack=False):
-    return HopProtocol(n_in, ticks, iters, s, b, max_ig, max_skip, weight_mode, on_round, backup_exact, notify_ack).run()
+             backup_exact=False, notify_ack=False, stale_reduce=NEW_ONLY):
+    return HopProtocol(n_in, ticks, iters, s, b, max_ig, max_skip, weight_mode, on_round, backup_exact, notify_ack,
+                       stale_reduce).run()
 
 
 # -------------------------------------------------------------------- graph helpers for the invariants

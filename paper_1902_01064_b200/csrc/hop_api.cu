@@ -60,6 +60,7 @@ struct hop_ctx {
     int32_t level = 0;
     std::vector<int32_t> newest;
     std::vector<std::vector<uint8_t>> sent;   // [N][level] worker entered (sent) that iteration
+    std::vector<int32_t> taken;               // per in-edge: newest version consumed over it (hop_step_host validation)
     int32_t* d_err = nullptr;
     int sm_count = 0;
     int64_t launches = 0;
@@ -118,6 +119,7 @@ extern "C" int hop_create(hop_ctx** out, const int32_t* in_ptr, const int32_t* i
     c->sp.b.assign(N, b);
     c->newest.assign(N, 0);
     c->sent.assign(N, {});
+    c->taken.assign(c->g.in_idx.size(), -1);
     *out = c;
     return HOP_OK;
 }
@@ -176,6 +178,11 @@ extern "C" int hop_set_option(hop_ctx* c, int key, double v) {
     if (key == HOP_OPT_APPROACH) {
         if (v != HOP_APPROACH_PARALLEL && v != HOP_APPROACH_SERIAL) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: unknown approach");
         c->serial = v == HOP_APPROACH_SERIAL;
+        return HOP_OK;
+    }
+    if (key == HOP_OPT_STALE_REDUCE) {
+        if (v != HOP_STALE_NEW_ONLY && v != HOP_STALE_REUSE) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: unknown stale-reduce mode");
+        c->sp.stale_reuse = v == HOP_STALE_REUSE;
         return HOP_OK;
     }
     if (key == HOP_OPT_BACKUP_MODE) {
@@ -354,10 +361,11 @@ extern "C" int hop_load_trace(hop_ctx* c, const hop_trace* t) {
     for (int32_t k = 0; k < L; ++k)
         for (int32_t i = 0; i < N; ++i) sent[i][k] = t->op[(size_t)k * N + i] == HOP_OP_NORMAL;
     std::vector<HopLevelHost> levels(L);
+    std::vector<int32_t> taken(c->g.in_idx.size(), -1);
     for (int32_t k = 0; k < L; ++k) {
         const size_t r = (size_t)k * N;
         const int rc = hop_validate_level(c->g, c->sp, k, &t->op[r], &t->ptr[r], t->nbr.data(), t->ver.data(),
-                                          t->num.data(), &t->den[r], newest, &sent, c->err);
+                                          t->num.data(), &t->den[r], newest, &sent, &taken, c->err);
         if (rc) return rc;
         hop_build_level(c->g, c->s, k, &t->op[r], &t->ptr[r], t->nbr.data(), t->ver.data(), t->num.data(), &t->den[r], levels[k]);
         const int rc2 = plan_level(c, levels[k]);
@@ -401,6 +409,7 @@ extern "C" int hop_load_trace(hop_ctx* c, const hop_trace* t) {
     c->mid_step = false;
     c->level = 0;
     std::fill(c->newest.begin(), c->newest.end(), 0);
+    std::fill(c->taken.begin(), c->taken.end(), -1);
     return HOP_OK;
 }
 
@@ -619,8 +628,8 @@ extern "C" int hop_step_host(hop_ctx* c, const int32_t* op, const int64_t* ptr, 
         if ((int32_t)c->sent[i].size() <= k) c->sent[i].resize(k + 1, 0);
         c->sent[i][k] = op[i] == HOP_OP_NORMAL;
     }
-    std::vector<int32_t> newest = c->newest;
-    rc = hop_validate_level(c->g, c->sp, k, op, ptr, nbr, ver, num, den, newest, &c->sent, c->err);
+    std::vector<int32_t> newest = c->newest, taken = c->taken;
+    rc = hop_validate_level(c->g, c->sp, k, op, ptr, nbr, ver, num, den, newest, &c->sent, &taken, c->err);
     if (rc) return rc;
     HopLevelHost L;
     hop_build_level(c->g, c->s, k, op, ptr, nbr, ver, num, den, L);
@@ -667,6 +676,7 @@ extern "C" int hop_step_host(hop_ctx* c, const int32_t* op, const int64_t* ptr, 
     rc = run_level(c, L, lv, TcPtrs{(const float*)(d + o_tcw), (const HopTcRow*)(d + o_tcr), (const int32_t*)(d + o_tcs)});
     if (rc) return rc;
     c->newest = newest;
+    c->taken.swap(taken);
     c->level += 1;
     if (probe_dst && probe_len > 0) {
         const float* src = c->X + ((int64_t)0 * (c->s + 1) + c->newest[0] % (c->s + 1)) * c->P;
@@ -681,6 +691,7 @@ extern "C" int hop_set_level(hop_ctx* c, int32_t level) {
     if (!c) return HOP_E_ARG;
     if (level < 0 || (c->loaded && level > (int32_t)c->levels.size())) HOP_FAIL(c, HOP_E_ARG, "hop_set_level: out of range");
     c->mid_step = false;
+    std::fill(c->taken.begin(), c->taken.end(), -1);    // hop_step_host's per-edge order check starts afresh
     // newest version held by each worker after levels [0, level)
     std::fill(c->newest.begin(), c->newest.end(), 0);
     if (c->loaded)

@@ -76,6 +76,7 @@ struct HopSimParams {
     int32_t s, max_ig /*0 = none*/, max_skip, weight_mode;
     int32_t notify_ack = 0;     // NOTIFY-ACK back-pressure (Section 3.3) instead of token queues
     int32_t backup_exact = 0;   // keep exactly |N_in| - b updates (own + earliest senders) instead of every usable one
+    int32_t stale_reuse = 0;    // 1: a usable update an earlier Recv already returned is reduced again (HOP_STALE_REUSE)
     std::vector<int32_t> b;
 };
 
@@ -86,7 +87,7 @@ int hop_simulate(const HopGraph& g, const HopSimParams& p, const uint64_t* ticks
 int hop_validate_level(const HopGraph& g, const HopSimParams& p, int32_t level, const int32_t* op,
                        const int64_t* ptr, const int32_t* nbr, const int32_t* ver, const int32_t* num,
                        const int32_t* den, std::vector<int32_t>& newest,
-                       std::vector<std::vector<uint8_t>>* sent, std::string& err);
+                       std::vector<std::vector<uint8_t>>* sent, std::vector<int32_t>* taken, std::string& err);
 void hop_build_level(const HopGraph& g, int32_t s, int32_t level, const int32_t* op, const int64_t* ptr,
                      const int32_t* nbr, const int32_t* ver, const int32_t* num, const int32_t* den,
                      HopLevelHost& out);

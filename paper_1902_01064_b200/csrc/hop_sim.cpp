@@ -8,6 +8,9 @@
 //     (one queue per iteration slot keeps newer ones out of reach, Section 6); it is usable iff
 //     v >= k - s (Section 4.4).  Recv completes once |N_in(i)| - N_buw(i) in-neighbours (self
 //     counts) are usable and then takes every usable one (Fig. alg4: needed + extras).
+//   * What a Recv dequeued is gone from the queue.  Under HOP_STALE_NEW_ONLY (Eq. 2's index set, Fig. alg3's
+//     test on what this call dequeued) a usable update enters the Reduce only if it is newer than the
+//     one the worker's previous Recv saw from that neighbour; one mark per in-edge keeps that.
 //   * TokenQ(j->i).size() = Iter(j) - Iter(i) + max_ig (proof of Theorem 2), so "a token is
 //     available from every out-neighbour" is Iter(j) >= Iter(i) + 1 - max_ig for all of them, and
 //     the straggler test of Section 5 (how many tokens the out-neighbours hold for me) is
@@ -30,6 +33,7 @@ struct Decision {
     enum Kind : int8_t { NONE, APPLIED, ENTER, PLAN_JUMP, JUMP } kind = NONE;
     int32_t target = 0;
     std::vector<std::pair<int32_t, int32_t>> got;   // (neighbour, version)
+    std::vector<int32_t> seen;                      // per in-edge of the worker: usable version this Recv saw, -1 none
 };
 
 struct Sim {
@@ -44,6 +48,7 @@ struct Sim {
     std::vector<int32_t> applied;                   // newest iteration whose Reduce/Apply is done (-1: none)
     std::vector<std::vector<int32_t>> entered;      // iterations a worker has entered, ascending
     std::vector<std::vector<int64_t>> entered_seq;  // global order of those Send events (arrival order at every receiver)
+    std::vector<int32_t> reduced;                   // per in-edge: newest version the receiver's completed Recvs have seen
     int64_t send_seq = 0;
     uint64_t now = 0;
     using Ev = std::pair<uint64_t, int32_t>;
@@ -54,7 +59,7 @@ struct Sim {
 
     Sim(const HopGraph& g_, const HopSimParams& p_, const uint64_t* t, int32_t it, hop_trace& o)
         : g(g_), p(p_), ticks(t), iters(it), N(g_.N), iter(N, 0), phase(N, COMPUTE), jump_to(N, 0), applied(N, -1),
-          entered(N), entered_seq(N), r_nbr((size_t)it * N), r_ver((size_t)it * N), r_num((size_t)it * N), out(o) {}
+          entered(N), entered_seq(N), reduced(g_.in_idx.size(), -1), r_nbr((size_t)it * N), r_ver((size_t)it * N), r_num((size_t)it * N), out(o) {}
 
     int32_t newest_entered_upto(int32_t j, int32_t level) const {
         const auto& e = entered[j];
@@ -73,11 +78,12 @@ struct Sim {
     bool try_recv(int32_t i, int32_t level, int32_t own_version, Decision& d) const {
         d.got.clear();
         const int32_t a = g.in_ptr[i], e = g.in_ptr[i + 1];
+        d.seen.assign(e - a, -1);
         for (int32_t t = a; t < e; ++t) {
             const int32_t j = g.in_idx[t];
             if (j == i && own_version >= 0) { d.got.push_back({j, own_version}); continue; }
             const int32_t v = newest_entered_upto(j, level);
-            if (v >= 0 && v >= level - p.s) d.got.push_back({j, v});
+            if (v >= 0 && v >= level - p.s) { d.got.push_back({j, v}); d.seen[t - a] = v; }
         }
         const int32_t need = (e - a) - p.b[i];
         if ((int32_t)d.got.size() < need) return false;
@@ -99,7 +105,22 @@ struct Sim {
             for (auto jv : d.got) if (keep[jv.first]) kept.push_back(jv);
             d.got.swap(kept);
         }
+        if (!p.stale_reuse) {
+            // only updates newer than what an earlier Recv of this worker already took out of the queue
+            std::vector<std::pair<int32_t, int32_t>> fresh;
+            for (auto jv : d.got) {
+                const int32_t t = (int32_t)(std::lower_bound(g.in_idx.begin() + a, g.in_idx.begin() + e, jv.first) - g.in_idx.begin());
+                if (jv.first == i || jv.second > reduced[t]) fresh.push_back(jv);
+            }
+            d.got.swap(fresh);
+        }
         return true;
+    }
+
+    void recv_done(int32_t i, const Decision& d) {
+        const int32_t a = g.in_ptr[i];
+        for (size_t t = 0; t < d.seen.size(); ++t)
+            if (d.seen[t] >= 0) reduced[a + t] = d.seen[t];
     }
 
     Decision decide(int32_t i) const {
@@ -195,6 +216,7 @@ struct Sim {
                     switch (d.kind) {
                     case Decision::APPLIED:
                         record(HOP_OP_NORMAL, k, i, d, -1);
+                        recv_done(i, d);
                         applied[i] = k;
                         if (p.notify_ack) touch_neighbours(i, next_dirty);   // an ACK may release an in-neighbour
                         if (k == iters - 1) { phase[i] = DONE; ++done; } else phase[i] = WAIT_TOKEN;
@@ -209,6 +231,7 @@ struct Sim {
                         break;
                     case Decision::JUMP:
                         record(HOP_OP_JUMP, d.target - 1, i, d, d.target - 1);
+                        recv_done(i, d);
                         enter(i, d.target);
                         touch_neighbours(i, next_dirty);
                         break;

@@ -54,11 +54,14 @@ extern "C" int hop_trace_destroy(hop_trace* t) { delete t; return HOP_OK; }
 
 // One level of records checked against the rules the protocol guarantees.  `newest[i]` is the
 // newest version worker i holds before the level and is advanced; `sent` (optional, [N][levels])
-// marks the iterations a worker entered, i.e. the versions other workers may consume.
+// marks the iterations a worker entered, i.e. the versions other workers may consume; `taken`
+// (optional, one per in-edge, -1 = nothing yet) is the newest version the receiver has consumed over
+// that edge and is advanced: a FIFO queue never hands out an older update after a newer one, and
+// under HOP_STALE_NEW_ONLY never the same one twice.
 int hop_validate_level(const HopGraph& g, const HopSimParams& p, int32_t level, const int32_t* op,
                        const int64_t* ptr, const int32_t* nbr, const int32_t* ver, const int32_t* num,
                        const int32_t* den, std::vector<int32_t>& newest,
-                       std::vector<std::vector<uint8_t>>* sent, std::string& err) {
+                       std::vector<std::vector<uint8_t>>* sent, std::vector<int32_t>* taken, std::string& err) {
     const int32_t N = g.N;
     auto fail = [&](int32_t i, const std::string& what) {
         err = "trace record (level " + std::to_string(level) + ", worker " + std::to_string(i) + "): " + what;
@@ -76,14 +79,18 @@ int hop_validate_level(const HopGraph& g, const HopSimParams& p, int32_t level, 
         if (o == HOP_OP_NORMAL && newest[i] != level) return fail(i, "NORMAL but the worker does not hold version " + std::to_string(level));
         if (o == HOP_OP_JUMP && !(newest[i] <= level && newest[i] >= level - p.s)) return fail(i, "JUMP but the held version is outside [k-s, k]");
         const int32_t d = g.in_ptr[i + 1] - g.in_ptr[i];
-        if (e - a < d - p.b[i]) return fail(i, "fewer than |N_in| - b consumed updates");
+        // Fig. alg4's count is about usable updates; with s > 0 and HOP_STALE_NEW_ONLY the Reduce may hold fewer
+        // (only the newly received ones, Eq. 2), down to the own update alone
+        const bool may_be_fewer = p.s > 0 && !p.stale_reuse;
+        if (!may_be_fewer && e - a < d - p.b[i]) return fail(i, "fewer than |N_in| - b consumed updates");
         if (e - a > d) return fail(i, "more consumed updates than in-neighbours");
         int64_t sum = 0;
         bool own = false;
         for (int64_t t = a; t < e; ++t) {
             const int32_t j = nbr[t], v = ver[t];
             if (j < 0 || j >= N) return fail(i, "neighbour id out of range");
-            if (!std::binary_search(g.in_idx.begin() + g.in_ptr[i], g.in_idx.begin() + g.in_ptr[i + 1], j))
+            const auto edge = std::lower_bound(g.in_idx.begin() + g.in_ptr[i], g.in_idx.begin() + g.in_ptr[i + 1], j);
+            if (edge == g.in_idx.begin() + g.in_ptr[i + 1] || *edge != j)
                 return fail(i, "consumed worker " + std::to_string(j) + " is not an in-neighbour");
             if (seen[j] == i) return fail(i, "neighbour consumed twice");
             seen[j] = i;
@@ -93,6 +100,13 @@ int hop_validate_level(const HopGraph& g, const HopSimParams& p, int32_t level, 
                 if (v != newest[i]) return fail(i, "own entry must name the version the worker holds");
             } else if (sent && !(*sent)[j][v]) {
                 return fail(i, "version " + std::to_string(v) + " of worker " + std::to_string(j) + " was never sent");
+            }
+            if (taken && j != i) {
+                int32_t& last = (*taken)[edge - g.in_idx.begin()];
+                if (v < last) return fail(i, "version " + std::to_string(v) + " of worker " + std::to_string(j) + " is older than one consumed before");
+                if (v == last && !p.stale_reuse)
+                    return fail(i, "version " + std::to_string(v) + " of worker " + std::to_string(j) + " was consumed before (HOP_STALE_NEW_ONLY reduces newly received updates only)");
+                last = v;
             }
             if (num[t] <= 0) return fail(i, "non-positive weight numerator");
             sum += num[t];

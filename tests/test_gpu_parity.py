@@ -1,7 +1,12 @@
 """Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element.
 
+The configurations run under both readings of the bounded-staleness Reduce set (only newly received updates, the
+default, as Eq. 2 and Fig. alg3 print it; or every update still inside the bound): `reduce` below.
+
 Tolerances (float32 path against a float64 oracle): max|delta| <= 1e-6 * max|x| after one level,
 <= 1e-4 * max|x| after a full run; traces are compared bit for bit."""
+import dataclasses
+
 import numpy as np
 import pytest
 import torch
@@ -70,7 +75,8 @@ def oracle_grad_fn(w, cols=None, external_G=None, loss="hinge"):
 
 def oracle_run(w, x0, levels, cols=None, external_G=None, variant=None):
     variant = variant or {}
-    tr = op.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode).to_arrays()
+    tr = op.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode,
+                     stale_reduce=w.stale_reduce).to_arrays()
     xs = x0.astype(np.float64) if cols is None else x0[:, cols].astype(np.float64)
     X, newest = up.run_updates(tr, w.N, w.lr, w.momentum, xs, oracle_grad_fn(w, cols, external_G, variant.get("loss", "hinge")),
                                levels=levels, s=w.s, weight_decay=variant.get("weight_decay", 0.0),
@@ -100,6 +106,11 @@ def check(w, levels, tol, mix_kernel=hop.MIX_AUTO, perturb=False, cols=None, ext
 
 
 KERNELS = [hop.MIX_STAGED, hop.MIX_BULK]
+REDUCE = [op.NEW_ONLY, op.REUSE]
+
+
+def workload(cfg, reduce=op.NEW_ONLY, **kw):
+    return dataclasses.replace(inputs.make_workload(cfg, **kw), stale_reduce=reduce)
 
 
 # ------------------------------------------------------------------ configuration 1: dense SVM, 4 workers
@@ -112,9 +123,10 @@ def test_cfg1_full_run_and_one_step(kernel):
 
 
 # ------------------------------------------------------------------ configuration 2: CSR SVM, 16 workers
+@pytest.mark.parametrize("reduce", REDUCE)
 @pytest.mark.parametrize("kernel", KERNELS)
-def test_cfg2_reduced_full_run(kernel):
-    w = inputs.make_workload(2, P=8192)
+def test_cfg2_reduced_full_run(kernel, reduce):
+    w = workload(2, reduce, P=8192)
     check(w, w.iters, TOL_RUN, kernel)
     check(w, 1, TOL_STEP, kernel, perturb=True)
 
@@ -126,10 +138,11 @@ def test_cfg2_full_size_first_levels():
 
 
 # ------------------------------------------------------------------ configuration 3: momentum + skipping
+@pytest.mark.parametrize("reduce", REDUCE)
 @pytest.mark.parametrize("kernel,P", [(hop.MIX_STAGED, 5000), (hop.MIX_BULK, 5000), (hop.MIX_STAGED, 4999),
                                       (hop.MIX_BULK, 132), (hop.MIX_STAGED, 3)])
-def test_cfg3_reduced_full_run(kernel, P):
-    w = inputs.make_workload(3, P=P)
+def test_cfg3_reduced_full_run(kernel, P, reduce):
+    w = workload(3, reduce, P=P)
     check(w, w.iters, TOL_RUN, kernel)
     check(w, 1, TOL_STEP, kernel, perturb=True)
 
@@ -145,9 +158,10 @@ def test_cfg3_full_size_sampled_columns():
 
 
 # ------------------------------------------------------------------ configuration 4: 64 workers, s=4, b=2
+@pytest.mark.parametrize("reduce", REDUCE)
 @pytest.mark.parametrize("kernel", KERNELS)
-def test_cfg4_reduced_full_run(kernel):
-    w = inputs.make_workload(4, P=3000)
+def test_cfg4_reduced_full_run(kernel, reduce):
+    w = workload(4, reduce, P=3000)
     check(w, w.iters, TOL_RUN, kernel)
     check(w, 1, TOL_STEP, kernel, perturb=True)
 
@@ -163,9 +177,10 @@ def test_cfg4_full_size_sampled_columns():
 
 
 # ------------------------------------------------------------------ configuration 5: complete graph, 128 workers
+@pytest.mark.parametrize("reduce", REDUCE)
 @pytest.mark.parametrize("kernel", KERNELS + [hop.MIX_TENSOR])
-def test_cfg5_reduced_full_run(kernel):
-    w = inputs.make_workload(5, P=1536)
+def test_cfg5_reduced_full_run(kernel, reduce):
+    w = workload(5, reduce, P=1536)
     g = GpuRun(w, kernel)
     assert g.h.level_stats(3)["kernel"] == kernel                      # the requested kernel is the one that runs
     g.h.close()
@@ -253,12 +268,14 @@ def test_in_place_ring_hazard_single_slot_and_stale_reads():
                             weight_mode=inputs.STALE_LINEAR, grad_mode=inputs.GRAD_SYNTHETIC, in_ptr=ptr, in_idx=idx,
                             ticks=ticks, grad_seed=77)
         w._p0 = rng.standard_normal(P).astype(np.float32)
-        tr = op.simulate(w.n_in, ticks, iters, s, 0, w.max_ig, 0, w.weight_mode)
-        if s > 0:
-            oldest = sum(1 for (k, i), rec in tr.rec.items() for (j, v, _) in rec if j != i and v == k - s)
-            assert oldest > 0, "no slot is read in the level that overwrites it: test is vacuous"
-        for kernel in KERNELS:
-            check(w, iters, TOL_RUN, kernel, perturb=True)
+        for reduce in (REDUCE if s > 0 else REDUCE[:1]):
+            w.stale_reduce = reduce
+            tr = op.simulate(w.n_in, ticks, iters, s, 0, w.max_ig, 0, w.weight_mode, stale_reduce=reduce)
+            if s > 0:
+                oldest = sum(1 for (k, i), rec in tr.rec.items() for (j, v, _) in rec if j != i and v == k - s)
+                assert oldest > 0, "no slot is read in the level that overwrites it: test is vacuous"
+            for kernel in KERNELS:
+                check(w, iters, TOL_RUN, kernel, perturb=True)
 
 
 @pytest.mark.parametrize("cfg,P,iters", [(3, 2048, 40), (5, 1536, 8)])
@@ -321,6 +338,15 @@ def test_malformed_traces_are_rejected_on_the_host():
     load(lambda t: t["den"].__setitem__((3, 3), t["den"][3, 3] + 1))          # weights do not sum up
     load(lambda t: t["op"].__setitem__((2, 0), 7))                            # unknown op
     g.h.load_trace(g.trace)
+    g.h.close()
+    # a trace that reduces an update again is valid only under HOP_STALE_REUSE
+    g = GpuRun(dataclasses.replace(w, stale_reduce=op.REUSE))
+    reused = g.trace
+    assert reused.dims()[2] > good["nbr"].size
+    g.h.set_option(hop.OPT_STALE_REDUCE, hop.STALE_NEW_ONLY)
+    with pytest.raises(hop.HopError) as e:
+        g.h.load_trace(reused)
+    assert e.value.code == hop.E_TRACE and "consumed before" in str(e.value)
     g.h.close()
 
 
@@ -466,7 +492,8 @@ def test_tensor_path_with_two_result_buffers(N, s, b):
     rng = np.random.default_rng(31)
     w = inputs.Workload(0, "dense-stale", N, P, iters, s=s, b=b, max_skip=0, max_ig=s, lr=0.05, momentum=0.0,
                         weight_mode=inputs.STALE_LINEAR, grad_mode=inputs.GRAD_SYNTHETIC, in_ptr=ptr, in_idx=idx,
-                        ticks=rng.choice([1, 2, 9], size=(N, iters)).astype(np.uint64), grad_seed=5)
+                        ticks=rng.choice([1, 2, 9], size=(N, iters)).astype(np.uint64), grad_seed=5,
+                        stale_reduce=op.REUSE)        # every update inside the bound is reduced: the widest contractions
     w._p0 = rng.standard_normal(P).astype(np.float32)
     g = GpuRun(w, hop.MIX_TENSOR)
     st = [g.h.level_stats(k) for k in range(iters)]

@@ -176,13 +176,88 @@ def test_staleness_window_and_gap(name, n_in, s):
                 for j in range(N):
                     if i != j:
                         assert p.Iter[i] - p.Iter[j] <= (s + 1) * dist[j][i]      # Table 1, row 2
-        tr = op.simulate(n_in, rand_ticks(rng, N, 12, 1, 30), 12, s=s, weight_mode=op.STALE_LINEAR, on_round=chk)
-        for (k, i), rec in tr.rec.items():
-            assert sorted(j for j, _, _ in rec) == sorted(n_in[i])               # b = 0: everyone
-            for (j, v, w) in rec:
-                assert k - s <= v <= k                                           # never older than s
-                assert w == v - (k - s) + 1                                      # Eq. 2 numerator
-            assert tr.den[(k, i)] == sum(w for _, _, w in rec)
+        T = rand_ticks(rng, N, 12, 1, 30)
+        for mode in (op.NEW_ONLY, op.REUSE):
+            tr = op.simulate(n_in, T, 12, s=s, weight_mode=op.STALE_LINEAR, on_round=chk, stale_reduce=mode)
+            for (k, i), rec in tr.rec.items():
+                if mode == op.REUSE:
+                    assert sorted(j for j, _, _ in rec) == sorted(n_in[i])       # b = 0: everyone, every level
+                else:
+                    assert (i, k, s + 1) in rec                                  # the own update is always new
+                    assert set(j for j, _, _ in rec) <= set(n_in[i])
+                for (j, v, w) in rec:
+                    assert k - s <= v <= k                                       # never older than s
+                    assert 1 <= w == v - (k - s) + 1 <= s + 1                    # Eq. 2 numerator
+                assert tr.den[(k, i)] == sum(w for _, _, w in rec)
+
+
+def _pairs(text):
+    return [tuple(int(x) for x in item.split(":")) for item in text.split(",")]
+
+
+def test_stale_reduce_hand_worked_example():
+    """Section 4.4 / Eq. 2 worked by hand (tests/golden): one neighbour stalls, its last update stays inside the
+    bound for two more iterations.  NEW_ONLY (Eq. 2's index set, Fig. alg3's `if`) leaves it out of those Reduces,
+    REUSE counts it again with a lower weight; both block and resume at the same tick."""
+    g = golden()
+    s = int(g["stale_example.s"])
+    ticks = np.ones((3, 6), np.uint64)
+    ticks[0, 1] = int(g["stale_example.slow_ticks"])
+    want = {op.NEW_ONLY: ("den_new_only", "consumed_new_only_iter2"), op.REUSE: ("den_reuse", "consumed_reuse_iter2")}
+    for mode, (kd, kc) in want.items():
+        entered = {}
+
+        def chk(p):
+            entered.setdefault((1, p.Iter[1]), p.now)
+        tr = op.simulate(inputs.complete(3), ticks, 6, s=s, b=0, max_ig=None, weight_mode=op.STALE_LINEAR,
+                         stale_reduce=mode, on_round=chk)
+        assert [tr.den[(k, 1)] for k in range(5)] == [int(x) for x in g["stale_example." + kd].split(",")]
+        assert [(j, v) for j, v, _ in tr.rec[(2, 1)]] == _pairs(g["stale_example." + kc])
+        assert entered[(1, 5)] == int(g["stale_example.release_tick_iter4"])    # Recv(4) completes, iteration 5 entered
+
+
+@pytest.mark.parametrize("s,b,max_ig,max_skip", [(1, 0, None, 0), (2, 0, 2, 0), (3, 1, 3, 0), (2, 1, 2, 2), (4, 2, 4, 0)])
+def test_new_only_is_reuse_minus_what_the_previous_recv_already_took(s, b, max_ig, max_skip):
+    """The two readings differ only in the Reduce set, never in when a Recv completes: same ops, same makespan, and a
+    NEW_ONLY record is the REUSE record without the (neighbour, iteration) pairs that the worker's previous Recv had
+    already returned.  (Derived here from the REUSE trace alone, independently of the oracle's bookkeeping.)"""
+    rng = np.random.default_rng(100 + s)
+    dropped = 0
+    for name, n_in in GRAPHS:
+        if any(b >= len(nb) for nb in n_in):
+            continue
+        N = len(n_in)
+        T = rand_ticks(rng, N, 14, 1, 25)
+        kw = dict(s=s, b=b, max_ig=max_ig, max_skip=max_skip, weight_mode=op.STALE_LINEAR)
+        new = op.simulate(n_in, T, 14, stale_reduce=op.NEW_ONLY, **kw)
+        old = op.simulate(n_in, T, 14, stale_reduce=op.REUSE, **kw)
+        assert np.array_equal(new.op, old.op) and new.makespan == old.makespan
+        for i in range(N):
+            prev = set()
+            for k in range(14):
+                if (k, i) not in old.rec:
+                    continue
+                full = [(j, v) for j, v, _ in old.rec[(k, i)]]
+                expect = [(j, v) for (j, v) in full if j == i or (j, v) not in prev]
+                assert [(j, v) for j, v, _ in new.rec[(k, i)]] == expect, (name, i, k)
+                nums, den = op.reduce_weights([k if j == i else v for j, v in expect], k, s, op.STALE_LINEAR)
+                assert [w for _, _, w in new.rec[(k, i)]] == nums and new.den[(k, i)] == den
+                dropped += len(full) - len(expect)
+                prev = set(full)
+    assert dropped > 0, "no neighbour ever stalled: the test is vacuous"
+
+
+def test_new_only_equals_reuse_when_nothing_is_stale():
+    """s = 0 (Figs. alg1 / alg4): an update of iteration k is first dequeued by Recv(k), so both readings coincide."""
+    rng = np.random.default_rng(17)
+    for name, n_in in GRAPHS:
+        for b in (0, 1):
+            if any(b >= len(nb) for nb in n_in):
+                continue
+            T = rand_ticks(rng, len(n_in), 10, 1, 20)
+            a = op.simulate(n_in, T, 10, s=0, b=b, max_ig=2, stale_reduce=op.NEW_ONLY).to_arrays()
+            c = op.simulate(n_in, T, 10, s=0, b=b, max_ig=2, stale_reduce=op.REUSE).to_arrays()
+            assert all(np.array_equal(a[k], c[k]) for k in a)
 
 
 def test_staleness_stuck_neighbour_reaches_s_plus_one():
@@ -264,11 +339,14 @@ def test_table1_last_row_with_tokens(s, b):
                     for j in range(N):
                         if i != j:
                             assert p.Iter[i] - p.Iter[j] <= min(b0 * dist[j][i], max_ig * dist[i][j])
-            tr = op.simulate(n_in, rand_ticks(rng, N, 10, 1, 25), 10, s=s, b=b, max_ig=max_ig,
-                             weight_mode=op.STALE_LINEAR, on_round=chk)
-            for (k, i), rec in tr.rec.items():
-                assert len(rec) >= len(n_in[i]) - b
-                assert all(k - s <= v <= k for _, v, _ in rec)
+            T = rand_ticks(rng, N, 10, 1, 25)
+            for mode in (op.NEW_ONLY, op.REUSE):
+                tr = op.simulate(n_in, T, 10, s=s, b=b, max_ig=max_ig, weight_mode=op.STALE_LINEAR, on_round=chk,
+                                 stale_reduce=mode)
+                for (k, i), rec in tr.rec.items():
+                    # the count rule of Fig. alg4 is about what is usable; NEW_ONLY may reduce fewer when s > 0
+                    assert len(rec) >= (len(n_in[i]) - b if (mode == op.REUSE or s == 0) else 1)
+                    assert all(k - s <= v <= k for _, v, _ in rec)
 
 
 # ------------------------------------------------------------------ skipping iterations

@@ -39,7 +39,8 @@ def _rank_main(rank, world, port, P, out):
     dist.init_process_group("gloo", rank=rank, world_size=world)
     w = inputs.make_workload(3, P=P, iters=12)
     lo, hi = bench.shard_columns(P, world, rank)
-    tr = op.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode).to_arrays()   # replicated
+    tr = op.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode,
+                           stale_reduce=w.stale_reduce).to_arrays()   # replicated
     cols = np.arange(lo, hi)
     x0 = np.tile(w.p0()[cols].astype(np.float64), (w.N, 1))
     X, newest = up.run_updates(tr, w.N, w.lr, w.momentum, x0, up.GradSynthetic(w.grad_seed, w.sigma, cols), s=w.s)
@@ -63,7 +64,8 @@ def test_two_ranks_reproduce_the_unsharded_run(tmp_path):
     mp.spawn(_rank_main, args=(2, _free_port(), P, out), nprocs=2, join=True)
     got = np.load(out)
     w = inputs.make_workload(3, P=P, iters=12)
-    tr = op.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode).to_arrays()
+    tr = op.simulate(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode,
+                           stale_reduce=w.stale_reduce).to_arrays()
     x0 = np.tile(w.p0().astype(np.float64), (w.N, 1))
     X, newest = up.run_updates(tr, w.N, w.lr, w.momentum, x0, up.GradSynthetic(w.grad_seed, w.sigma, np.arange(P)), s=w.s)
     want = np.stack([X[(i, newest[i])] for i in range(w.N)])

@@ -11,7 +11,7 @@ from paper_1902_01064_b200 import hop, inputs
 KEYS = ("op", "ptr", "nbr", "ver", "num", "den")
 
 
-def both(n_in, ticks, iters, s, b, max_ig, max_skip, mode, exact=False, notify_ack=False):
+def both(n_in, ticks, iters, s, b, max_ig, max_skip, mode, exact=False, notify_ack=False, reduce=op.NEW_ONLY):
     ptr, idx = inputs.graph_to_csr(n_in)
     n_in = inputs.csr_to_lists(ptr, idx)                 # records list neighbours in ascending id order
     h = hop.Hop(ptr, idx, len(n_in), 8, s, b, max_skip)
@@ -19,9 +19,11 @@ def both(n_in, ticks, iters, s, b, max_ig, max_skip, mode, exact=False, notify_a
     h.set_option(hop.OPT_WEIGHT_MODE, mode)
     h.set_option(hop.OPT_BACKUP_MODE, hop.BACKUP_EXACT if exact else hop.BACKUP_AT_LEAST)
     h.set_option(hop.OPT_NOTIFY_ACK, 1 if notify_ack else 0)
+    assert (hop.STALE_NEW_ONLY, hop.STALE_REUSE) == (op.NEW_ONLY, op.REUSE)
+    h.set_option(hop.OPT_STALE_REDUCE, reduce)
     got = h.sim_run(ticks, iters).to_arrays()
     want_tr = op.simulate(n_in, ticks, iters, s, b, None if notify_ack else max_ig, max_skip, mode, backup_exact=exact,
-                          notify_ack=notify_ack)
+                          notify_ack=notify_ack, stale_reduce=reduce)
     want = want_tr.to_arrays()
     h.close()
     return got, want, want_tr.makespan
@@ -33,12 +35,17 @@ def assert_same(got, want, makespan, ctx=""):
     assert got["makespan"] == makespan, ctx
 
 
+@pytest.mark.parametrize("reduce", [op.NEW_ONLY, op.REUSE])
 @pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
-def test_configs_bit_exact(cfg):
+def test_configs_bit_exact(cfg, reduce):
     w = inputs.make_workload(cfg, P=64 if cfg == 1 else 256)
-    got, want, mk = both(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode)
+    got, want, mk = both(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode, reduce=reduce)
     assert_same(got, want, mk, cfg)
     assert (got["op"] != op.IDLE).sum() > 0
+    if reduce == op.NEW_ONLY:      # every configuration has stalled neighbours: the two readings must differ
+        other = both(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode, reduce=op.REUSE)[0]
+        assert np.array_equal(other["op"], got["op"]) and other["makespan"] == got["makespan"]
+        assert other["ptr"][-1] > got["ptr"][-1]
 
 
 def _enumerate(name, n_in, iters, values, combos):
@@ -50,8 +57,9 @@ def _enumerate(name, n_in, iters, values, combos):
             if any(b >= len(nb) for nb in n_in) or max_skip > s + 1:
                 continue
             max_ig = max(1, s)
-            got, want, mk = both(n_in, ticks, iters, s, b, max_ig, max_skip, op.STALE_LINEAR)
-            assert_same(got, want, mk, (name, flat, s, b, max_skip))
+            for reduce in ((op.NEW_ONLY, op.REUSE) if s > 0 else (op.NEW_ONLY,)):    # the readings coincide at s = 0
+                got, want, mk = both(n_in, ticks, iters, s, b, max_ig, max_skip, op.STALE_LINEAR, reduce=reduce)
+                assert_same(got, want, mk, (name, flat, s, b, max_skip, reduce))
             count += 1
     return count
 
@@ -105,8 +113,9 @@ def test_random_graphs_long_runs_with_ties_and_skips():
                 h.sim_run(ticks, iters)
             assert e.value.code == hop.E_DEADLOCK
             continue
-        got, want, mk = both(n_in, ticks, iters, s, b, max_ig, max_skip, mode)
-        assert_same(got, want, mk, trial)
+        for reduce in (op.NEW_ONLY, op.REUSE):
+            got, want, mk = both(n_in, ticks, iters, s, b, max_ig, max_skip, mode, reduce=reduce)
+            assert_same(got, want, mk, (trial, reduce))
 
 
 def test_unbounded_gap_without_tokens():
@@ -131,32 +140,41 @@ def test_exact_backup_mode_bit_exact_and_exactly_d_minus_b():
         max_skip = int(rng.integers(0, s + 2)) if trial % 2 else 0
         iters = 20
         ticks = rng.choice([1, 2, 3, 9], size=(N, iters)).astype(np.uint64)
-        try:
-            got, want, mk = both(n_in, ticks, iters, s, b, 3, max_skip, op.STALE_LINEAR, exact=True)
-        except op.Deadlock:
-            continue
-        assert_same(got, want, mk, trial)
-        cnt = np.diff(got["ptr"]).reshape(iters, N)
-        for i in range(N):
-            active = got["op"][:, i] != op.IDLE
-            assert (cnt[active, i] == len(n_in[i]) - b).all()          # exactly in-degree - b consumed
+        for reduce in (op.REUSE, op.NEW_ONLY):
+            try:
+                got, want, mk = both(n_in, ticks, iters, s, b, 3, max_skip, op.STALE_LINEAR, exact=True, reduce=reduce)
+            except op.Deadlock:
+                continue
+            assert_same(got, want, mk, (trial, reduce))
+            cnt = np.diff(got["ptr"]).reshape(iters, N)
+            for i in range(N):
+                active = got["op"][:, i] != op.IDLE
+                if reduce == op.REUSE or s == 0:
+                    assert (cnt[active, i] == len(n_in[i]) - b).all()      # exactly in-degree - b consumed
+                else:
+                    assert (cnt[active, i] >= 1).all() and (cnt[active, i] <= len(n_in[i]) - b).all()
     for name, n_in in inputs.small_cases():
         if name.endswith("3"):
             continue
         for flat in itertools.product((1, 2, 3), repeat=8):
             ticks = np.asarray(flat, np.uint64).reshape(4, 2)
-            got, want, mk = both(n_in, ticks, 2, 1, 1, 1, 0, op.UNIFORM, exact=True)
-            assert_same(got, want, mk, (name, flat))
+            for reduce in (op.REUSE, op.NEW_ONLY):
+                got, want, mk = both(n_in, ticks, 2, 1, 1, 1, 0, op.UNIFORM, exact=True, reduce=reduce)
+                assert_same(got, want, mk, (name, flat, reduce))
 
 
+@pytest.mark.parametrize("reduce", [op.REUSE, op.NEW_ONLY])
 @pytest.mark.parametrize("cfg", [2, 4, 5])
-def test_configs_bit_exact_in_exact_backup_mode(cfg):
+def test_configs_bit_exact_in_exact_backup_mode(cfg, reduce):
     w = inputs.make_workload(cfg, P=256)
-    got, want, mk = both(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode, exact=True)
+    got, want, mk = both(w.n_in, w.ticks, w.iters, w.s, w.b, w.max_ig, w.max_skip, w.weight_mode, exact=True, reduce=reduce)
     assert_same(got, want, mk, cfg)
     d = np.diff(w.in_ptr)
     cnt = np.diff(got["ptr"]).reshape(w.iters, w.N)
-    assert (cnt == (d - w.b)[None, :]).all()
+    if reduce == op.REUSE:
+        assert (cnt == (d - w.b)[None, :]).all()
+    else:
+        assert (cnt >= 1).all() and (cnt <= (d - w.b)[None, :]).all() and (cnt < (d - w.b)[None, :]).any()
 
 
 def test_notify_ack_bit_exact():
