@@ -29,11 +29,11 @@ if ROOT not in sys.path:
 METRIC = "worker_iterations_per_s"
 UNIT = "worker-iterations/s"
 PROBE = 1024
-# dram__bytes_read.sum + dram__bytes_write.sum (bytes, per launch, averaged over the trace) of the mix-update kernel
-# from the ncu captures summarised under profiles/: taken at a smaller parameter count and scaled by the number of
-# columns (traffic is proportional to columns at a fixed trace).  Dropped to None whenever the kernel changes.
-NCU_TRAFFIC = {(4, 25_600_000): 23.49e9,      # profiles/mix_bulk_kernel_cfg4.md, section 2b (all 50 levels, current kernel)
-               (5, 8_000_000): 12.64e9}       # profiles/mix_dense_tc_kernel_cfg5.md, section 2b (all 30 levels, current kernel)
+# dram__bytes_read.sum + dram__bytes_write.sum of the mix-update kernel, one value per level of the trace, from an ncu
+# capture at a smaller parameter count P (same trace; traffic grows in proportion to the columns).  bench_config sums
+# it over exactly the levels the timed region ran and scales by columns.  An entry is removed whenever its kernel, the
+# trace or the gradient kernel in front of it changes.
+NCU_LEVEL_TRAFFIC = {}
 
 
 def shard_columns(P: int, n: int, r: int, unit: int = 128):
@@ -88,6 +88,14 @@ class ClockSampler(threading.Thread):
             except Exception:
                 pass
             time.sleep(0.02)
+
+    def sample_now(self):
+        if self.nv is None:
+            return
+        try:
+            self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.dev, self.nv.NVML_CLOCK_SM))
+        except Exception:
+            pass
 
     def result(self):
         if not self.samples:
@@ -196,41 +204,41 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", type=int, default=4)
-    ap.add_argument("--impl", default="ours")
-    ap.add_argument("--P", type=int, default=None, help="override the parameter count (profiling on a small case)")
-    ap.add_argument("--mix-kernel", type=int, default=0)
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--graph", default="auto", choices=["auto", "0", "1"],
-                    help="timed region replays CUDA graphs of the trace (hop_run); auto = only for small, launch-bound workloads")
-    args = ap.parse_args()
-    if args.impl == "reference":
-        return run_reference(args)
-
+def measure_tf32_peak(dev):
+    """Dense TF32 matmul throughput of this GPU, measured the way the bf16 figure in MEASURED_PEAKS.json was: an
+    8192^3 library matmul (TF32 tensor cores allowed), best of 10, CUDA events.  A denominator only; not on the path."""
     import torch
-    from paper_1902_01064_b200 import build as _b
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if rank == 0:
-        _b.build()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the Hop hot path has no CPU fallback")
-    torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-        dist.barrier()
-    from paper_1902_01064_b200 import hop, inputs
+    old = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = True
+    try:
+        n = 8192
+        a = torch.randn((n, n), dtype=torch.float32, device=dev)
+        b = torch.randn((n, n), dtype=torch.float32, device=dev)
+        c = torch.empty((n, n), dtype=torch.float32, device=dev)
+        for _ in range(3):
+            torch.matmul(a, b, out=c)
+        best = float("inf")
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            torch.matmul(a, b, out=c)
+            e1.record()
+            e1.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        del a, b, c
+        return 2.0 * n ** 3 / (best * 1e-3) / 1e12
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = old
 
-    w = inputs.make_workload(args.config, P=args.P)
+
+def bench_config(args, cfg, env):
+    """Times `args.steps` levels of configuration `cfg` on this rank's column shard and returns the result dict
+    (rank 0: the JSON fields; other ranks: None)."""
+    import torch
+    from paper_1902_01064_b200 import hop, inputs
+    world, rank, local, dist = env["world"], env["rank"], env["local"], env["dist"]
+    steps = args.steps
+    w = inputs.make_workload(cfg, P=args.P)
     P_global = w.P
     lo, hi = shard_columns(P_global, world, rank)
     p0 = w.p0()[lo:hi].copy()
@@ -265,7 +273,7 @@ def main():
     tr = trace.to_arrays()
     wi_per_level = (tr["op"] == 1).sum(axis=1)
     stats = [h.level_stats(k) for k in range(w.iters)]
-    timed = {"flops": 0}
+    timed = {"flops": 0, "levels": []}
     p0_dev = torch.from_numpy(p0).to(dev)
 
     def reset():
@@ -304,6 +312,7 @@ def main():
                 h.step()
             wi += int(wi_per_level[k:k + m].sum())
             timed["flops"] += sum(st["mma_flops"] for st in stats[k:k + m])
+            timed["levels"].extend(range(k, k + m))
             k += m
             done += m
         return wi
@@ -313,7 +322,7 @@ def main():
     run_levels(max(3, args.warmup))
     if use_graph:                      # instantiate the graphs outside the timed region
         reset()
-        run_levels(args.steps, graph=True)
+        run_levels(steps, graph=True)
     reset()
     barrier()
     sampler = ClockSampler(local)
@@ -322,10 +331,11 @@ def main():
     h.timing_enable(not use_graph)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    timed["flops"] = 0
-    wi = run_levels(args.steps, graph=use_graph)
-    mma_flops = timed["flops"]
+    timed["flops"], timed["levels"] = 0, []
+    wi = run_levels(steps, graph=use_graph)
+    mma_flops, timed_levels = timed["flops"], list(timed["levels"])
     e1.record(stream)
+    sampler.sample_now()               # short runs end between two periodic samples: take one while the work is in flight
     barrier()
     sampler.stop_flag = True
     ms = e0.elapsed_time(e1)
@@ -333,7 +343,7 @@ def main():
     if use_graph:                      # per-kernel event timing is not possible inside a replayed graph: separate pass
         reset()
         h.timing_enable(True)
-        run_levels(args.steps)
+        run_levels(steps)
         torch.cuda.synchronize()
     tim = h.timing_read()
     h.timing_enable(False)
@@ -360,7 +370,7 @@ def main():
                               np.ascontiguousarray(tr["nbr"][a:b]), np.ascontiguousarray(tr["ver"][a:b]),
                               np.ascontiguousarray(tr["num"][a:b]), np.ascontiguousarray(tr["den"][k])))
         probe = np.zeros(min(PROBE, w.P), np.float32)
-        n_e2e = min(args.steps, w.iters)
+        n_e2e = min(steps, w.iters)
         for k in range(min(3, w.iters)):
             h.step_host(*per_level[k], probe)
         reset()
@@ -376,55 +386,141 @@ def main():
             t = torch.tensor([t_e2e], dtype=torch.float64, device=dev)
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             t_e2e = float(t.item())
+
         def table_bytes(st):      # what hop_step_host copies to the device for one level
             b = st["U"] * 4 + st["normal"] * 4 + (st["normal"] + st["jump"]) * 32 + st["entries"] * 8
             if st["kernel"] == hop.MIX_TENSOR:
                 b += st["k_padded"] * 512 + 128 * 12 + st["k_padded"] * 4
             return b
-        h2d = float(np.mean([table_bytes(h.level_stats(k)) for k in range(n_e2e)]))
+        h2d = float(np.mean([table_bytes(stats[k]) for k in range(n_e2e)]))
         e2e = {"value": wi2 / t_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 4.0 * min(PROBE, w.P),
                "steps": n_e2e, "note": "hop_step_host: level records from host memory through a pinned staging buffer, "
                "probe of worker 0 read back, stream synchronised every step"}
 
+    ring_bytes = X.numel() * 4
+    h.close()
+    del X, M, G, keep, p0_dev
+    torch.cuda.empty_cache()
     if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return
+        return None
     peak, bf16_peak, peak_kind = measured_peaks()
     kernels = sorted({st["kernel"] for st in stats})
     kname = {hop.MIX_STAGED: "mix_staged_kernel", hop.MIX_BULK: "mix_bulk_kernel", hop.MIX_TENSOR: "mix_dense_tc_kernel"}
     mix_launches = tim["spans"][1]
-    ach = tim["mix_bytes"] / (tim["ms_mix"] * 1e-3) / 1e9 if tim["ms_mix"] > 0 else 0.0
-    traffic = NCU_TRAFFIC.get((args.config, P_global))
+    mix_s = tim["ms_mix"] * 1e-3
+    ach = tim["mix_bytes"] / mix_s / 1e9 if mix_s > 0 else 0.0
+    alg_per_launch = tim["mix_bytes"] / max(1, mix_launches)
+    # measured DRAM traffic of exactly the levels that were timed (ncu on a smaller parameter count, scaled by columns)
+    traffic = None
+    cap = NCU_LEVEL_TRAFFIC.get(cfg)
+    if (cap is not None and args.P is None and args.mix_kernel == 0 and w.stale_reduce == cap["stale_reduce"]
+            and len(cap["bytes"]) == w.iters and mix_launches == len(timed_levels)):
+        traffic = float(np.mean([cap["bytes"][k] for k in timed_levels])) * (w.P / cap["P"])
     roofline = {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
-                "traffic": traffic, "traffic_unit": "bytes per launch", "peak_kind": f"of {peak_kind}", "kernel": "+".join(kname[k] for k in kernels),
+                "traffic": traffic, "traffic_unit": "bytes per launch",
+                "traffic_over_alg": (traffic / alg_per_launch) if traffic and alg_per_launch else None,
+                "dram_frac": (traffic / (mix_s / max(1, mix_launches)) / 1e9 / peak) if traffic and mix_s > 0 else None,
+                "peak_kind": f"of {peak_kind}", "kernel": "+".join(kname[k] for k in kernels),
                 "kernel_timing": ("separate step-by-step pass with per-kernel events (the timed region replays CUDA graphs)"
                                   if use_graph else "CUDA events inside the timed region"),
                 "launches": mix_launches, "avg_launch_ms": tim["ms_mix"] / max(1, mix_launches),
-                "alg_bytes_per_launch": tim["mix_bytes"] / max(1, mix_launches),
+                "alg_bytes_per_launch": alg_per_launch,
                 "frac_of_nominal_8TBs": ach / 8000.0,
+                "note": ("frac is algorithmic bytes / time / copy bandwidth: the freshly written gradient rows are partly still in "
+                         "L2 when the mix reads them, so DRAM traffic is below the algorithmic bytes and frac can pass 1; "
+                         "dram_frac is the measured traffic / time / the same peak"),
                 "other_kernels_ms": {"gradient": tim["ms_grad"], "sparse_apply": tim["ms_apply"]}}
+    if ring_bytes <= 3e8:
+        roofline["note"] = "the ring fits the 126 MB L2 (or nearly): absolute numbers only, frac is not an HBM fraction"
     if hop.MIX_TENSOR in kernels:
-        # tensor-pipe view of the same launches: two TF32 MMA passes over K padded to 32; TF32 peak = the measured
-        # bf16 matmul peak times the nominal TF32/bf16 ratio (1.1 / 2.25 PFLOP/s)
-        flops = mma_flops
-        tf32_peak = bf16_peak * 1.1 / 2.25
-        tf = flops / (tim["ms_mix"] * 1e-3) / 1e12 if tim["ms_mix"] > 0 else 0.0
-        roofline["tensor"] = {"achieved": tf, "peak": tf32_peak, "unit": "TFLOP/s", "frac": tf / tf32_peak, "dtype": "tf32 (2-pass split)",
-                              "note": "HBM binds: the contraction has ~%.0f flop per algorithmic byte" % (flops / max(1, tim["mix_bytes"]))}
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
-            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+        # tensor-pipe view of the same launches: two TF32 MMA passes over K padded to 32
+        tf32_derived = bf16_peak * 1.1 / 2.25
+        try:
+            tf32_peak, tf32_kind = measure_tf32_peak(dev), "measured tf32 (library matmul 8192^3, best of 10, this run)"
+        except Exception as ex:       # the denominator must never take the bench line down
+            tf32_peak, tf32_kind = tf32_derived, f"derived (measurement failed: {ex!r})"
+        tf = mma_flops / mix_s / 1e12 if mix_s > 0 else 0.0
+        roofline["tensor"] = {"achieved": tf, "peak": tf32_peak, "unit": "TFLOP/s", "frac": tf / tf32_peak, "peak_kind": tf32_kind,
+                              "peak_derived": tf32_derived, "peak_derived_kind": f"{peak_kind} bf16 peak x 1.1/2.25 (nominal ratio)",
+                              "dtype": "tf32 (2-pass split)",
+                              "note": "HBM binds: the contraction has ~%.0f flop per algorithmic byte" % (mma_flops / max(1, tim["mix_bytes"]))}
+    normal_timed = int(sum(int(wi_per_level[k]) for k in timed_levels))
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": max(3, args.warmup),
+            "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": f"config {args.config}: {w.name}", "N": w.N, "P": P_global, "P_per_gpu": w.P, "s": w.s, "b": w.b,
-                       "levels": w.iters, "trace_passes": args.steps / w.iters, "parallelism": f"column-sharded x{world}",
-                       "l2": "inputs exceed L2 (ring %.1f GB per GPU)" % (X.numel() * 4 / 1e9) if X.numel() * 4 > 3e8 else "ring fits L2: absolute numbers only",
+            "value_mix_only": (normal_timed / mix_s) if mix_s > 0 else None,
+            "config": {"workload": f"config {cfg}: {w.name}", "N": w.N, "P": P_global, "P_per_gpu": w.P, "s": w.s, "b": w.b,
+                       "levels": w.iters, "trace_passes": steps / w.iters, "parallelism": f"column-sharded x{world}",
+                       "stale_reduce": "new_only (Eq. 2 as printed)" if w.stale_reduce == 0 else "reuse",
+                       "timed_levels": f"{timed_levels[0]}..{timed_levels[-1]}" if steps <= w.iters else f"whole trace x{steps / w.iters:.2f}",
+                       "l2": "inputs exceed L2 (ring %.1f GB per GPU)" % (ring_bytes / 1e9) if ring_bytes > 3e8 else "ring fits L2: absolute numbers only",
                        "protocol_sim_ms": sim_ms,
                        "launch": "hop_run: CUDA graph replay of the trace" if use_graph else "hop_step per level"},
             "roofline": roofline, "gpu_launches": int(launches), "clocks": sampler.result()}
     if e2e is not None:
         line["e2e"] = e2e
-    if not args.no_cpu_baseline and world == 1:
-        wf = inputs.make_workload(args.config, P=args.P)
+    return line
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=None, help="1..5; default: 4 as the headline, then 5, 3, 2, 1 as `secondary`")
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"], help="process-group backend when WORLD_SIZE > 1")
+    ap.add_argument("--P", type=int, default=None, help="override the parameter count (profiling on a small case)")
+    ap.add_argument("--mix-kernel", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true")
+    ap.add_argument("--graph", default="auto", choices=["auto", "0", "1"],
+                    help="timed region replays CUDA graphs of the trace (hop_run); auto = only for small, launch-bound workloads")
+    args = ap.parse_args()
+    headline_cfg = 4 if args.config is None else args.config
+    if args.impl == "reference":
+        args.config = headline_cfg
+        return run_reference(args)
+
+    import torch
+    from paper_1902_01064_b200 import build as _b
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if rank == 0:
+        _b.build()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the Hop hot path has no CPU fallback")
+    n_dev = torch.cuda.device_count()
+    local = local % n_dev              # more ranks than devices (a test on one GPU): ranks share devices
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        if args.backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group("gloo")
+        dist.barrier()
+    from paper_1902_01064_b200 import inputs
+    env = {"world": world, "rank": rank, "local": local, "dist": dist}
+    if dist is not None and args.backend == "gloo":
+        env["dist"] = _HostCollectives(dist, torch.device("cuda", local))
+
+    line = bench_config(args, headline_cfg, env)
+    if rank == 0 and args.config is None and world == 1 and not args.no_secondary and args.P is None:
+        # the other configurations, same steps: compact records (no CPU baseline)
+        line["secondary"] = []
+        for cfg in (5, 3, 2, 1):
+            try:
+                r = bench_config(args, cfg, env)
+                line["secondary"].append({k: r[k] for k in ("config", "value", "value_mix_only", "unit", "steps", "ms_per_step",
+                                                             "roofline", "clocks", "gpu_launches", "e2e") if k in r})
+            except Exception as ex:       # a secondary record must never take the headline down
+                line["secondary"].append({"config": {"workload": f"config {cfg}"}, "error": repr(ex)})
+    if rank == 0 and not args.no_cpu_baseline and world == 1:
+        wf = inputs.make_workload(headline_cfg, P=args.P)
         v, desc = oracle_sample(wf)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
         try:
@@ -436,9 +532,31 @@ def main():
             line["cpu_baseline"]["all_cores"] = {"value": allc[0], "unit": UNIT, "cores": allc[1],
                                                  "sample": f"same update rules on {allc[2]} columns dealt to {allc[1]} processes "
                                                            f"({allc[3]:.2f} s), protocol simulation serial"}
-    print(json.dumps(line))
+    if rank == 0:
+        print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+class _HostCollectives:
+    """barrier / all_reduce for device tensors over a CPU process group (gloo): the tensor goes through host memory.
+    Only for running several ranks where NCCL cannot be used (ranks sharing one GPU in a test)."""
+
+    def __init__(self, dist, dev):
+        self.dist, self.dev, self.ReduceOp = dist, dev, dist.ReduceOp
+
+    def barrier(self):
+        self.dist.barrier()
+
+    def all_reduce(self, t, op=None):
+        import torch
+        torch.cuda.current_stream().synchronize()
+        host = t.detach().cpu()
+        self.dist.all_reduce(host, op=op if op is not None else self.dist.ReduceOp.SUM)
+        t.copy_(host.to(t.device))
+
+    def destroy_process_group(self):
+        self.dist.destroy_process_group()
 
 
 if __name__ == "__main__":

@@ -145,6 +145,13 @@ int hop_create(hop_ctx** out, const int32_t* in_ptr, const int32_t* in_idx,
                int32_t N, int64_t P, int32_t s, int32_t b, int32_t max_skip);
 int hop_destroy(hop_ctx* ctx);
 const char* hop_last_error(const hop_ctx* ctx);
+/* Options may be set at any time except between hop_step_begin and hop_step_end.  Every call drops the CUDA
+ * graphs hop_run has cached.  With a trace loaded, a change of HOP_OPT_MOMENTUM (zero <-> non-zero),
+ * HOP_OPT_WEIGHT_DECAY (zero <-> non-zero), HOP_OPT_APPROACH, HOP_OPT_GRAD_MODE or HOP_OPT_MIX_KERNEL plans and
+ * uploads the loaded levels again (tile widths, kernel choice and the staged rows depend on them; this frees and
+ * allocates the device tables and synchronises) and keeps the current level; if the trace cannot be planned
+ * under the new value the call fails and the option keeps its old value.  The protocol options (max_ig, weight
+ * mode, backup mode, stale-reduce mode, N_buw) act on hop_sim_run and on the validation of traces loaded later. */
 int hop_set_option(hop_ctx* ctx, int key, double value);
 
 /* ---- protocol simulation (host only, no GPU) --------------------------------------------------
@@ -175,7 +182,9 @@ int hop_bind_buffers(hop_ctx* ctx, float* X, float* M, float* G, void* cuda_stre
  * coef_r = -y_r / batch if y_r * margin_r < 1 else 0; g = sum_r coef_r a_r.  The minibatch of
  * iteration k is rows [(k mod (rows_per_worker/batch)) * batch, +batch) of the worker's shard.
  * Dense: A[N][rows_per_worker][P], y[N][rows_per_worker] (device).  CSR: row_ptr[N*rows+1]
- * (global offsets), col, val, y (device).  Allocates N*batch floats of device scratch. */
+ * (global offsets), col, val, y (device).  Allocates N*batch floats of device scratch (a second bind frees
+ * and reallocates it, synchronising the device, and drops the CUDA graphs hop_run has cached, since they hold
+ * the old pointers). */
 int hop_bind_svm_dense(hop_ctx* ctx, const float* A, const float* y,
                        int32_t rows_per_worker, int32_t batch);
 int hop_bind_svm_csr(hop_ctx* ctx, const int64_t* row_ptr, const int32_t* col, const float* val,

@@ -53,6 +53,7 @@ struct hop_ctx {
     HopRecord* d_rec = nullptr;
     HopEntry* d_ent = nullptr;
     bool loaded = false;
+    hop_trace loaded_trace;         // host copy: the levels are planned again when an option that shapes the plan changes
     // streaming mode (hop_step_host): pinned staging + device copy of one level
     void* h_stage = nullptr; void* d_stage = nullptr; size_t stage_cap = 0;
     float* h_probe = nullptr; size_t probe_cap = 0;
@@ -159,10 +160,7 @@ extern "C" int hop_destroy(hop_ctx* c) {
     return HOP_OK;
 }
 
-extern "C" int hop_set_option(hop_ctx* c, int key, double v) {
-    if (!c) return HOP_E_ARG;
-    if (!std::isfinite(v)) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: the value must be finite");
-    drop_graphs(c);
+static int set_option_value(hop_ctx* c, int key, double v) {
     if (key == HOP_OPT_USE_GRAPH) { c->use_graph = v != 0.0; return HOP_OK; }
     if (key == HOP_OPT_NOTIFY_ACK) { c->sp.notify_ack = v != 0.0; return HOP_OK; }
     if (key == HOP_OPT_WEIGHT_DECAY) {
@@ -225,6 +223,43 @@ extern "C" int hop_set_option(hop_ctx* c, int key, double v) {
     return HOP_OK;
 }
 
+static int load_trace_impl(hop_ctx* c, const hop_trace& t, bool rewind);
+
+// What plan_level bakes into a loaded level: staged rows, tile width, kernel choice, the gradient rows of the dense path.
+struct PlanShape {
+    bool mom, decay, serial; int32_t grad_mode, mix_kernel;
+    bool operator==(const PlanShape& o) const {
+        return mom == o.mom && decay == o.decay && serial == o.serial && grad_mode == o.grad_mode && mix_kernel == o.mix_kernel;
+    }
+};
+static PlanShape plan_shape(const hop_ctx* c) {
+    return PlanShape{c->momentum != 0.0, c->weight_decay != 0.0, c->serial, c->grad_mode, c->mix_kernel};
+}
+
+extern "C" int hop_set_option(hop_ctx* c, int key, double v) {
+    if (!c) return HOP_E_ARG;
+    if (!std::isfinite(v)) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: the value must be finite");
+    if (c->mid_step) HOP_FAIL(c, HOP_E_STATE, "hop_set_option: a hop_step_begin is waiting for its hop_step_end");
+    drop_graphs(c);
+    const PlanShape before = plan_shape(c);
+    const double old_mom = c->momentum, old_wd = c->weight_decay;
+    const bool old_serial = c->serial;
+    const int32_t old_gm = c->grad_mode, old_mk = c->mix_kernel;
+    const int rc = set_option_value(c, key, v);
+    if (rc) return rc;
+    if (c->loaded && !(plan_shape(c) == before)) {
+        // the loaded levels were planned for the old setting: plan and upload them again, keeping the position
+        const int rr = load_trace_impl(c, c->loaded_trace, false);
+        if (rr) {            // not plannable under the new setting: keep the old one (tables untouched)
+            const std::string why = c->err;
+            c->momentum = old_mom; c->weight_decay = old_wd; c->serial = old_serial; c->grad_mode = old_gm; c->mix_kernel = old_mk;
+            c->err = "hop_set_option: the loaded trace cannot be planned with this value (" + why + "); option unchanged";
+            return rr;
+        }
+    }
+    return HOP_OK;
+}
+
 extern "C" int hop_sim_run(hop_ctx* c, const uint64_t* ticks, int32_t iters, hop_trace** out) {
     if (!c || !ticks || !out || iters <= 0) { if (c) c->err = "hop_sim_run: bad argument"; return HOP_E_ARG; }
     hop_trace* t = new hop_trace;
@@ -261,6 +296,8 @@ static int alloc_coef(hop_ctx* c, int32_t R, int32_t B) {
     if (R <= 0 || B <= 0 || R % B != 0) HOP_FAIL(c, HOP_E_ARG, "SVM shard: rows_per_worker must be a positive multiple of batch");
     const int rc = ensure_device(c);
     if (rc) return rc;
+    drop_graphs(c);      // captured kernels hold the old scratch and data pointers
+    if (c->mid_step) HOP_FAIL(c, HOP_E_STATE, "SVM shard: a hop_step_begin is waiting for its hop_step_end");
     if (c->coef) { cudaFree(c->coef); c->coef = nullptr; }
     if (c->margins) { cudaFree(c->margins); c->margins = nullptr; }
     HOP_CUDA(c, cudaMalloc(&c->coef, (size_t)c->g.N * B * sizeof(float)));
@@ -355,6 +392,12 @@ extern "C" int hop_load_trace(hop_ctx* c, const hop_trace* t) {
     if (!c || !t) return HOP_E_ARG;
     if (!c->bound) HOP_FAIL(c, HOP_E_STATE, "hop_load_trace: bind buffers first");
     if (t->N != c->g.N) HOP_FAIL(c, HOP_E_TRACE, "hop_load_trace: trace has a different number of workers");
+    return load_trace_impl(c, *t, true);
+}
+
+// Validates, plans and uploads; rewind = false keeps the current level (the same trace planned again).
+static int load_trace_impl(hop_ctx* c, const hop_trace& trace, bool rewind) {
+    const hop_trace* t = &trace;
     const int32_t N = t->N, L = t->levels;
     std::vector<int32_t> newest(N, 0);
     std::vector<std::vector<uint8_t>> sent(N, std::vector<uint8_t>(L, 0));
@@ -407,9 +450,12 @@ extern "C" int hop_load_trace(hop_ctx* c, const hop_trace* t) {
     c->sent = std::move(sent);
     c->loaded = true;
     c->mid_step = false;
-    c->level = 0;
-    std::fill(c->newest.begin(), c->newest.end(), 0);
-    std::fill(c->taken.begin(), c->taken.end(), -1);
+    if (&trace != &c->loaded_trace) c->loaded_trace = trace;
+    if (rewind) {
+        c->level = 0;
+        std::fill(c->newest.begin(), c->newest.end(), 0);
+        std::fill(c->taken.begin(), c->taken.end(), -1);
+    }
     return HOP_OK;
 }
 
@@ -463,18 +509,20 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, c
     cfg.sm_count = c->sm_count; cfg.err_word = c->d_err; cfg.stream = c->stream;
     cfg.table_smem = L.table_smem; cfg.n_ents = (int32_t)L.ents.size();
     int e = 0;
+    bool grad_kernel_in_front = false;      // a gradient kernel of this library was launched by this call, right before the mix
     if (L.nG > 0 && c->grad_mode != HOP_GRAD_EXTERNAL) {
         HOP_SPAN_BEGIN();
         switch (c->grad_mode) {
         case HOP_GRAD_SYNTHETIC:
-            if (phase != 2) { e = hop_launch_synth_grad(cfg, lv, c->grad_seed, (float)c->sigma, c->col_offset); c->launches += 1; }
+            if (phase != 2) { e = hop_launch_synth_grad(cfg, lv, c->grad_seed, (float)c->sigma, c->col_offset); c->launches += 1; grad_kernel_in_front = true; }
             break;
         case HOP_GRAD_SVM_DENSE:
             e = hop_launch_svm_dense(cfg, lv, c->svmA, c->svmY, c->svmR, c->svmB, c->coef, c->margins, phase);
-            c->launches += phase == 1 ? 1 : 2; break;
+            c->launches += (phase == 1 || (phase == 0 && hop_svm_dense_is_fused(c->P, c->svmB))) ? 1 : 2;
+            grad_kernel_in_front = true; break;
         case HOP_GRAD_SVM_CSR:
             e = hop_launch_svm_csr_coef(cfg, lv, c->svmRowPtr, c->svmCol, c->svmVal, c->svmY, c->svmR, c->svmB, c->coef, c->margins, phase);
-            c->launches += 1; break;
+            c->launches += 1; grad_kernel_in_front = true; break;
         default: break;
         }
         if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("gradient kernel launch: ") + cudaGetErrorString((cudaError_t)e));
@@ -491,7 +539,11 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, c
         if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("apply launch: ") + cudaGetErrorString((cudaError_t)e));
         HOP_SPAN_END(2, 0);
         cfg.use_g = 0; cfg.mu = 0.f; cfg.wd = 0.f;      // the mix only averages
+        grad_kernel_in_front = false;                   // the apply kernel in front writes X
     }
+    // None of the gradient kernels writes X or M, and each was launched with a full dependency on everything before it:
+    // the mix may fetch its X and M rows while such a kernel drains (it waits before it reads G and before it stores).
+    cfg.early_x = grad_kernel_in_front ? 1 : 0;
     if (L.nA > 0) {
         HOP_SPAN_BEGIN();
         if (L.kernel == HOP_MIX_TENSOR)

@@ -125,6 +125,8 @@ struct HopLaunchCfg {
     int32_t* err_word;  // device
     int32_t table_smem; // bytes of shared memory holding the level's records + entries (0 = read from global)
     int32_t n_ents;
+    int32_t early_x;    // the mix launch may overlap the tail of the gradient kernel launched just before it (which writes
+                        // neither X nor M): programmatic dependent launch
     void* stream;
 };
 int hop_launch_mix_staged(const HopLaunchCfg& c, const HopLevelDev& lv);
@@ -140,6 +142,7 @@ int hop_launch_svm_csr_apply(const HopLaunchCfg& c, const HopLevelDev& lv, const
                              const float* val, int32_t R, int32_t B, const float* coef, int32_t slot_shift);
 // serial approach, dense gradients: x_k <- x_k - lr * d in place for the level's NORMAL workers
 int hop_launch_apply_dense(const HopLaunchCfg& c, const HopLevelDev& lv);
+bool hop_svm_dense_is_fused(int64_t P, int32_t B);   // the dense SVM gradient of a level is one launch instead of two
 int hop_mix_smem_budget(int kernel);   // usable dynamic shared memory per CTA for the kernel
 int hop_mix_stages(int kernel);
 int hop_mix_table_limit();

@@ -224,6 +224,13 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
+// Programmatic dependent launch (PTX griddepcontrol): a kernel launched with the programmatic-serialization attribute may
+// start while the kernel in front of it in the stream is still running, once every block of that kernel has executed
+// launch_dependents (or exited); dependency_wait then blocks until that kernel has completed and its writes are visible.
+// Without the attribute, or with nothing in front, both are no-ops.
+__device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // A record as the bulk kernel keeps it in shared memory: everything that does not depend on the tile is worked out
 // once per block (the generic record costs ~60 instructions per tile and record in address arithmetic and flags).
 struct alignas(16) BulkRec {
@@ -290,11 +297,15 @@ __device__ __forceinline__ void bulk_record(const BulkRec& r, const int4* __rest
 // every staged row of the next tile, rows dealt round-robin to the producer lanes, completion counted
 // in bytes on an mbarrier), the other kConsumerWarps warps consume.  Two stages.
 // Requires P % 4 == 0 and 16-byte aligned base pointers (bulk copies move multiples of 16 bytes).
+// early_x != 0: the launch carries the programmatic-serialization attribute and the kernel in front of it in the stream
+// (the level's gradient kernel) writes neither X nor M: barrier set-up, the tables and the X / M rows of the first
+// kBulkStages tiles are then fetched while that kernel is still draining; the gradient rows and every store come
+// after dependency_wait.  early_x == 0: everything comes after it.
 template <bool MOMENTUM, bool DECAY>
 __global__ void __launch_bounds__(kBulkThreads, 1)
 mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __restrict__ G, int64_t P, int w,
                 int use_g, float lr, float mu, float lam, HopLevelDev lv, int table_bytes, int n_ents,
-                int32_t* __restrict__ err_word) {
+                int32_t* __restrict__ err_word, int early_x) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw);
     uint64_t* empty = full + kBulkStages;
@@ -308,6 +319,7 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
     const int rows = lv.U + nG * (MOMENTUM ? 2 : 1);
     const int64_t stage_floats = (int64_t)rows * w;
     const int64_t tiles = (P + w - 1) / w;
+    if (!early_x) dependency_wait();
     if (tid == 0) {
         for (int s = 0; s < kBulkStages; ++s) { mbar_init(&full[s], kProducerWarps); mbar_init(&empty[s], kConsumerWarps); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -335,21 +347,38 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
         }
         int64_t n = 0;
         bool ok = true;
-        for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++n) {
-            const int s = (int)(n % kBulkStages);
-            const uint32_t ph = (uint32_t)((n / kBulkStages) & 1);
-            if (!mbar_wait<256>(&empty[s], ph ^ 1u)) { ok = false; if (lane == 0) atomicCAS(err_word, 0, ERR_EMPTY_WAIT | (int)(tile & 0xffffff)); break; }
+        // which == 0: every row of this lane; 1: all but the gradient rows; 2: the gradient rows only
+        auto issue = [&](int64_t tile, int s, int which) {
             const int64_t c0 = tile * w;
             const int wd = (int)min((int64_t)w, P - c0);
             const uint32_t bytes = (uint32_t)wd * 4u;
-            if (lane == 0) mbar_expect_tx(&full[s], bytes * (uint32_t)my_rows);
-            __syncwarp();
+            if (which != 2) {
+                if (lane == 0) mbar_expect_tx(&full[s], bytes * (uint32_t)my_rows);
+                __syncwarp();
+            }
             float* dst = stage0 + s * stage_floats;
+            auto wanted = [&](int r) { return which == 0 || ((r >= lv.U && r < lv.U + nG) == (which == 2)); };
 #pragma unroll
-            for (int h = 0; h < kHoist; ++h)
-                if (src_h[h]) bulk_g2s(dst + (warp + (lane + 32 * h) * kProducerWarps) * w, src_h[h] + c0, bytes, &full[s]);
+            for (int h = 0; h < kHoist; ++h) {
+                const int r = warp + (lane + 32 * h) * kProducerWarps;
+                if (src_h[h] && wanted(r)) bulk_g2s(dst + r * w, src_h[h] + c0, bytes, &full[s]);
+            }
             for (int r = warp + (lane + 32 * kHoist) * kProducerWarps; r < rows; r += 32 * kProducerWarps)
-                bulk_g2s(dst + (int64_t)r * w, row_src(r) + c0, bytes, &full[s]);
+                if (wanted(r)) bulk_g2s(dst + (int64_t)r * w, row_src(r) + c0, bytes, &full[s]);
+        };
+        int64_t tile = blockIdx.x;
+        if (early_x) {
+            // the first tiles' X and M rows while the gradient kernel may still be writing G (both stages are free)
+            int pre = 0;
+            for (int64_t t = tile; t < tiles && pre < kBulkStages; t += gridDim.x, ++pre) issue(t, pre, 1);
+            dependency_wait();
+            for (int q = 0; q < pre; ++q, tile += gridDim.x, ++n) issue(tile, q, 2);
+        }
+        for (; tile < tiles && ok; tile += gridDim.x, ++n) {
+            const int s = (int)(n % kBulkStages);
+            const uint32_t ph = (uint32_t)((n / kBulkStages) & 1);
+            if (!mbar_wait<256>(&empty[s], ph ^ 1u)) { ok = false; if (lane == 0) atomicCAS(err_word, 0, ERR_EMPTY_WAIT | (int)(tile & 0xffffff)); break; }
+            issue(tile, s, 0);
         }
         // drain: do not leave while copies into this block's shared memory are still in flight
         if (ok) {
@@ -383,6 +412,7 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
             for (int i = ct; i < n_ents; i += kConsumerThreads) sent[i] = ge[i];
             asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
         }
+        if (early_x) dependency_wait();      // no store before the kernel in front has finished (it may read the slot written here)
         int64_t n = 0;
         for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++n) {
             const int s = (int)(n % kBulkStages);
@@ -446,6 +476,7 @@ __device__ __forceinline__ void box_muller(uint32_t ra, uint32_t rb, float sigma
 constexpr int kGradChunks = 4;
 __global__ void __launch_bounds__(256)
 synth_grad_kernel(float* __restrict__ G, int64_t P, HopLevelDev lv, uint32_t k0, uint32_t k1, float sigma, int64_t col_offset) {
+    launch_dependents();      // the mix-update kernel behind may set itself up; it waits before it touches G
     const int worker = lv.grad_workers[blockIdx.y];
     float* row = G + (int64_t)worker * P;
     const bool vec = (P & 3) == 0;
@@ -494,6 +525,7 @@ __global__ void __launch_bounds__(256)
 svm_margin_csr_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelDev lv, const int64_t* __restrict__ row_ptr,
                       const int32_t* __restrict__ col, const float* __restrict__ val, const float* __restrict__ y,
                       int R, int B, int loss, float* __restrict__ coef, double* __restrict__ margins_out) {
+    launch_dependents();
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (gw >= lv.nG * B) return;
     const int a = gw / B, r = gw - a * B;
@@ -513,6 +545,7 @@ svm_margin_csr_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelDev
 __global__ void __launch_bounds__(256)
 svm_coef_from_margins_kernel(const double* __restrict__ margins, HopLevelDev lv, const float* __restrict__ y, int R, int B,
                              int loss, float* __restrict__ coef) {
+    launch_dependents();
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= lv.nG * B) return;
     const int a = t / B, r = t - a * B;
@@ -545,6 +578,7 @@ svm_margin_dense_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelD
 __global__ void __launch_bounds__(256)
 svm_dense_grad_kernel(float* __restrict__ G, int64_t P, HopLevelDev lv, const float* __restrict__ A, int R, int B,
                       const float* __restrict__ coef) {
+    launch_dependents();
     const int worker = lv.grad_workers[blockIdx.y];
     const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (p >= P) return;
@@ -561,6 +595,43 @@ svm_dense_grad_kernel(float* __restrict__ G, int64_t P, HopLevelDev lv, const fl
     }
     for (; r < B; ++r) g = fmaf(cf[r], a0[(int64_t)r * P], g);
     G[(int64_t)worker * P + p] = g;
+}
+
+// Margins, coefficients and gradient of one worker's minibatch in one block (small problems: the three steps as separate
+// launches cost more in launch latency than in work).  Same arithmetic in the same order as svm_margin_dense_kernel
+// followed by svm_dense_grad_kernel: a warp per row for the margins, a thread per column for the gradient.
+constexpr int kFusedSvmThreads = 256;
+__global__ void __launch_bounds__(kFusedSvmThreads)
+svm_dense_fused_kernel(const float* __restrict__ X, float* __restrict__ G, int64_t P, int S, HopLevelDev lv,
+                       const float* __restrict__ A, const float* __restrict__ y, int R, int B, int loss) {
+    extern __shared__ float s_coef[];      // [B]
+    launch_dependents();
+    const int worker = lv.grad_workers[blockIdx.x];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row0 = (int64_t)worker * R + (int64_t)(lv.level % (R / B)) * B;
+    const float* x = X + ((int64_t)worker * S + lv.level % S) * P;
+    for (int r = warp; r < B; r += kFusedSvmThreads / 32) {
+        const float* arow = A + (row0 + r) * P;
+        double m = 0.0;
+        for (int64_t p = lane; p < P; p += 32) m += (double)arow[p] * (double)x[p];
+        m = warp_sum(m);
+        if (lane == 0) s_coef[r] = loss_coefficient(y[row0 + r], m, B, loss);
+    }
+    __syncthreads();
+    for (int64_t p = threadIdx.x; p < P; p += kFusedSvmThreads) {
+        const float* a0 = A + row0 * P + p;
+        float g = 0.f;
+        int r = 0;
+        for (; r + 8 <= B; r += 8) {
+            float a[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) a[i] = a0[(int64_t)(r + i) * P];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) g = fmaf(s_coef[r + i], a[i], g);
+        }
+        for (; r < B; ++r) g = fmaf(s_coef[r], a0[(int64_t)r * P], g);
+        G[(int64_t)worker * P + p] = g;
+    }
 }
 
 // Sparse Apply after the dense mix: x_{k+1,i}[col] -= lr * coef_r * val, one warp per row.
@@ -621,6 +692,9 @@ size_t staged_smem(const HopLaunchCfg& c, const HopLevelDev& lv) {
 
 }  // namespace
 
+// One launch for margins + coefficients + gradient when a worker's minibatch is small (B * P floats, read twice).
+bool hop_svm_dense_is_fused(int64_t P, int32_t B) { return B <= 4096 && (int64_t)B * P <= 65536; }
+
 int hop_mix_smem_budget(int kernel) { return kernel == HOP_MIX_BULK ? (227 * 1024 - 128) : 200 * 1024; }
 int hop_mix_table_limit() { return 32 * 1024; }
 int hop_mix_stages(int kernel) { return kernel == HOP_MIX_BULK ? kBulkStages : kStagedStages; }
@@ -661,12 +735,19 @@ int hop_launch_mix_bulk(const HopLaunchCfg& c, const HopLevelDev& lv) {
     const int grid = (int)std::min<int64_t>(tiles, (int64_t)c.sm_count);
     cudaStream_t st = (cudaStream_t)c.stream;
     cudaError_t e = cudaSuccess;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3((unsigned)grid); lc.blockDim = dim3(kBulkThreads); lc.dynamicSmemBytes = smem; lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = c.early_x ? 1 : 0;
 #define HOP_LAUNCH_BULK(MO, DE)                                                                               \
     do {                                                                                                      \
         e = hop_allow_max_smem<mix_bulk_kernel<MO, DE>>();                                                    \
         if (e == cudaSuccess)                                                                                 \
-            mix_bulk_kernel<MO, DE><<<grid, kBulkThreads, smem, st>>>(c.X, c.M, c.G, c.P, c.tile_w, c.use_g, c.lr, c.mu, c.wd, lv, \
-                                                                      c.table_smem, c.n_ents, c.err_word);   \
+            e = cudaLaunchKernelEx(&lc, mix_bulk_kernel<MO, DE>, c.X, c.M, (const float*)c.G, c.P, (int)c.tile_w, (int)c.use_g, c.lr, c.mu, \
+                                   c.wd, lv, (int)c.table_smem, (int)c.n_ents, c.err_word, (int)c.early_x);  \
     } while (0)
     const bool mom = c.mu != 0.f, dec = c.wd != 0.f;
     if (mom && dec) HOP_LAUNCH_BULK(true, true);
@@ -693,6 +774,10 @@ int hop_launch_svm_dense(const HopLaunchCfg& c, const HopLevelDev& lv, const flo
     if (lv.nG == 0) return 0;
     const int warps = lv.nG * B;
     cudaStream_t st = (cudaStream_t)c.stream;
+    if (phase == 0 && hop_svm_dense_is_fused(c.P, B)) {
+        svm_dense_fused_kernel<<<lv.nG, kFusedSvmThreads, (size_t)B * sizeof(float), st>>>(c.X, c.G, c.P, c.s + 1, lv, A, y, R, B, c.loss);
+        return (int)cudaGetLastError();
+    }
     if (phase != 2)
         svm_margin_dense_kernel<<<(warps * 32 + 255) / 256, 256, 0, st>>>(c.X, c.P, c.s + 1, lv, A, y, R, B, c.loss, coef,
                                                                           phase == 1 ? margins : nullptr);

@@ -585,3 +585,97 @@ def test_split_phase_calls_must_alternate():
     g.h.step()
     assert g.h.read_status() == 0
     g.h.close()
+
+
+# ------------------------------------------------------------------ options and data changed after the trace was loaded
+def _oracle_state(w, x0, levels, variant=None):
+    tr, want, newest = oracle_run(w, x0, levels, variant=variant)
+    return want, max(np.abs(x).max() for x in want)
+
+
+def test_options_set_after_load_trace_plan_the_levels_again():
+    # momentum switched on and off after the load: the staged rows and the tile width depend on it
+    w = workload(3, P=2048, iters=30)
+    x0 = np.stack([w.p0() + w.perturbation(i) for i in range(w.N)])
+    for late_mu in (0.9, 0.0):
+        g = GpuRun(w, x0=x0)                                   # planned with momentum 0.9, buffer bound
+        g.h.set_option(hop.OPT_MOMENTUM, 0.9 - late_mu)       # planned again with the other setting ...
+        g.h.set_option(hop.OPT_MOMENTUM, late_mu)             # ... and once more with the one that runs
+        got = g.run(w.iters)
+        want, scale = _oracle_state(dataclasses.replace(w, momentum=late_mu), x0, w.iters)
+        assert max(np.abs(got[i] - want[i]).max() for i in range(w.N)) <= TOL_RUN * scale
+        g.h.close()
+    # tensor path: serial order and weight decay chosen after the load (the dense path bakes its gradient rows in)
+    w = workload(5, P=1536, iters=8)
+    x0 = np.stack([w.p0() + w.perturbation(i) for i in range(w.N)])
+    g = GpuRun(w, hop.MIX_TENSOR, x0=x0)
+    assert g.h.level_stats(2)["kernel"] == hop.MIX_TENSOR
+    g.h.set_option(hop.OPT_APPROACH, hop.APPROACH_SERIAL)
+    assert g.h.level_stats(2)["kernel"] == hop.MIX_TENSOR
+    got = g.run(w.iters)
+    want, scale = _oracle_state(w, x0, w.iters, variant=dict(serial=True))
+    assert max(np.abs(got[i] - want[i]).max() for i in range(w.N)) <= TOL_RUN * scale
+    g.h.close()
+    g = GpuRun(w, hop.MIX_TENSOR, x0=x0)
+    g.h.set_option(hop.OPT_WEIGHT_DECAY, 0.05)                 # the dense path has no weight decay: another kernel takes over
+    assert g.h.level_stats(2)["kernel"] == hop.MIX_BULK
+    got = g.run(w.iters)
+    want, scale = _oracle_state(w, x0, w.iters, variant=dict(weight_decay=0.05))
+    assert max(np.abs(got[i] - want[i]).max() for i in range(w.N)) <= TOL_RUN * scale
+    # a value the loaded trace cannot be planned with is refused and leaves the context as it was
+    g.h.close()
+    w = workload(3, P=4999, iters=6)
+    g = GpuRun(w, hop.MIX_STAGED)
+    with pytest.raises(hop.HopError) as e:
+        g.h.set_option(hop.OPT_MIX_KERNEL, hop.MIX_BULK)       # needs P % 4 == 0
+    assert e.value.code == hop.E_UNSUPPORTED
+    assert g.h.level_stats(1)["kernel"] == hop.MIX_STAGED
+    g.h.step()
+    assert g.h.read_status() == 0
+    g.h.close()
+
+
+def test_option_change_in_the_middle_of_a_run_keeps_the_position():
+    w = workload(3, P=1024, iters=20)
+    x0 = np.stack([w.p0() + w.perturbation(i) for i in range(w.N)])
+    ref = GpuRun(w, x0=x0).run(w.iters)
+    g = GpuRun(w, x0=x0)
+    g.run(9)
+    g.h.set_option(hop.OPT_MIX_KERNEL, hop.MIX_STAGED)        # planned again at level 9
+    assert g.h.level_stats(12)["kernel"] == hop.MIX_STAGED
+    got = g.run(w.iters - 9)
+    for i in range(w.N):
+        assert g.h.newest_version(i) in (w.iters, w.iters - 1, w.iters - 2)
+        assert np.abs(got[i] - ref[i]).max() <= 1e-6 * np.abs(ref[i]).max()
+    g.h.close()
+
+
+@pytest.mark.parametrize("cfg,P,iters", [(1, None, 20), (2, 4096, 16)])
+def test_svm_rebind_between_graph_replays_uses_the_new_buffers(cfg, P, iters):
+    # hop_run caches CUDA graphs whose kernels hold the SVM data and scratch pointers: binding other buffers must
+    # drop them.  The old buffers are zeroed after the rebind, so a stale graph would show.
+    w = workload(cfg, P=P, iters=iters)
+    ref = GpuRun(w).run(w.iters)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        g = GpuRun(w)
+        g.h.run(w.iters)
+        side.synchronize()
+        if cfg == 1:
+            A2, y2 = g.A.clone(), g.y.clone()
+            g.h.bind_svm_dense(A2, y2, w.svm.rows_per_worker, w.svm.batch)
+            g.A.zero_(); g.y.zero_()
+        else:
+            new = [t.clone() for t in (g.rp, g.col, g.val, g.y)]
+            g.h.bind_svm_csr(*new, w.svm.rows_per_worker, w.svm.batch)
+            g.val.zero_(); g.y.zero_()
+        for i in range(w.N):
+            g.h.write_params(i, 0, g.x0[i])
+        g.h.set_level(0)
+        g.h.run(w.iters)
+        got = [g.h.read_params(i) for i in range(w.N)]
+        assert g.h.read_status() == 0
+    for i in range(w.N):
+        scale = np.abs(ref[i]).max() + 1e-30
+        assert np.abs(got[i] - ref[i]).max() <= 1e-5 * scale
+    g.h.close()
