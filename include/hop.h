@@ -90,7 +90,9 @@ typedef enum hop_loss { HOP_LOSS_HINGE = 0, HOP_LOSS_LOG = 1 } hop_loss;
 
 /* Order of the five operations inside an iteration (Section 3.2).  PARALLEL: Send x_k, Compute on x_k, Recv,
  * Reduce, Apply: x_{k+1} = Reduce(versions) - eta * d.  SERIAL: Compute, Apply, Send, Recv, Reduce:
- * x'_k = x_k - eta * d replaces version k in the ring before anyone consumes it, x_{k+1} = Reduce(versions). */
+ * x'_k = x_k - eta * d replaces version k in the ring before anyone consumes it, x_{k+1} = Reduce(versions).
+ * hop_sim_run follows the same order: in the serial approach the update of iteration k becomes visible to the
+ * out-neighbours when Compute(k) ends, in the parallel approach when iteration k is entered. */
 typedef enum hop_approach { HOP_APPROACH_PARALLEL = 0, HOP_APPROACH_SERIAL = 1 } hop_approach;
 
 /* Where the gradient of a level comes from. */

@@ -31,6 +31,9 @@ Readings taken where the paper is silent (listed once more in the design notes):
       required number, then whatever else is there), subject to R2'.  b = 0 is Fig. alg3, s = 0 is
       Fig. alg4 (an update of iteration k is first dequeued by Recv(k), so R2' changes nothing
       there), both 0 is Fig. alg1; both > 0 is the "hybrid" row of Table 1.
+  R3' serial=True is the serial approach of Section 3.2 (Compute, Apply, Send, Recv, Reduce): the update of
+      iteration k is enqueued when Compute(k) ends, not when the iteration is entered; tokens are still inserted
+      at the start of the iteration (Fig. alg2).  The default is the parallel approach the paper adopts.
   R4  Same-tick ordering: rounds.  In a round every worker decides its transition from the
       state left by the previous round; then all decisions are committed in worker order.
       One transition per worker per round; rounds repeat until nothing moves.
@@ -112,8 +115,9 @@ def reduce_weights(vers, level, s, weight_mode):
 class HopProtocol:
     def __init__(self, n_in, ticks, iters, s=0, b=0, max_ig=None, max_skip=0,
                  weight_mode=UNIFORM, on_round=None, backup_exact=False, notify_ack=False,
-                 stale_reduce=NEW_ONLY):
+                 stale_reduce=NEW_ONLY, serial=False):
         self.N = N = len(n_in)
+        self.serial = serial
         self.n_in = [list(nb) for nb in n_in]
         for i, nb in enumerate(self.n_in):
             if i not in nb:
@@ -162,16 +166,20 @@ class HopProtocol:
         self.trace = Trace(N, iters, np.zeros((iters, N), np.int32))
 
     # ---------------------------------------------------------------- paper operations
-    def _enter(self, i, k, n_tokens=1):
-        """Start of iteration k at worker i (Fig. alg2): insert tokens, Send, start Compute."""
-        if self.max_ig is not None:
-            for j in self.n_in[i]:
-                if j != i:
-                    self.token_q[(i, j)].extend([k] * n_tokens)
+    def _send(self, i, k):
         for j in self.n_out[i]:
             self.update_q[j].append((k, i))                     # UpdateQ(j).enqueue(x_{k,i}, iter=k, w_id=i)
             self.arrival_pos.setdefault((i, j), {})[k] = self.arrivals[j]
             self.arrivals[j] += 1
+
+    def _enter(self, i, k, n_tokens=1):
+        """Start of iteration k at worker i (Fig. alg2): insert tokens, Send (parallel approach), start Compute."""
+        if self.max_ig is not None:
+            for j in self.n_in[i]:
+                if j != i:
+                    self.token_q[(i, j)].extend([k] * n_tokens)
+        if not self.serial:
+            self._send(i, k)
         self.Iter[i] = k
         self.phase[i] = _COMPUTE
         self.end[i] = self.now + int(self.ticks[i][k])
@@ -195,7 +203,7 @@ class HopProtocol:
         for j in self.n_in[i]:
             if j == i and own_version is not None:
                 got.append((j, own_version))                     # jumper's current parameters
-            elif self.iter_rcv[(j, i)] >= level - self.s:
+            elif self.iter_rcv[(j, i)] >= max(level - self.s, 0):         # -1: nothing received from j yet (Fig. alg3)
                 got.append((j, self.iter_rcv[(j, i)]))
         need = len(self.n_in[i]) - self.b[i]
         if len(got) < need:
@@ -300,6 +308,8 @@ class HopProtocol:
             self.now = min(self.end[i] for i in computing)
             for i in computing:
                 if self.end[i] == self.now:
+                    if self.serial:
+                        self._send(i, self.Iter[i])               # Compute, Apply, then Send (Section 3.2)
                     self.phase[i] = _RECV
             while True:
                 acts = [(i, self._decide(i)) for i in range(self.N)]
@@ -315,9 +325,9 @@ class HopProtocol:
 
 
 def simulate(n_in, ticks, iters, s=0, b=0, max_ig=None, max_skip=0, weight_mode=UNIFORM, on_round=None,
-             backup_exact=False, notify_ack=False, stale_reduce=NEW_ONLY):
+             backup_exact=False, notify_ack=False, stale_reduce=NEW_ONLY, serial=False):
     return HopProtocol(n_in, ticks, iters, s, b, max_ig, max_skip, weight_mode, on_round, backup_exact, notify_ack,
-                       stale_reduce).run()
+                       stale_reduce, serial).run()
 
 
 # -------------------------------------------------------------------- graph helpers for the invariants

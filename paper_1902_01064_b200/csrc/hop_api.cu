@@ -176,6 +176,7 @@ static int set_option_value(hop_ctx* c, int key, double v) {
     if (key == HOP_OPT_APPROACH) {
         if (v != HOP_APPROACH_PARALLEL && v != HOP_APPROACH_SERIAL) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: unknown approach");
         c->serial = v == HOP_APPROACH_SERIAL;
+        c->sp.serial_send = c->serial ? 1 : 0;
         return HOP_OK;
     }
     if (key == HOP_OPT_STALE_REDUCE) {

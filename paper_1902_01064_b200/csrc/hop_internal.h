@@ -76,6 +76,7 @@ struct HopSimParams {
     int32_t s, max_ig /*0 = none*/, max_skip, weight_mode;
     int32_t notify_ack = 0;     // NOTIFY-ACK back-pressure (Section 3.3) instead of token queues
     int32_t backup_exact = 0;   // keep exactly |N_in| - b updates (own + earliest senders) instead of every usable one
+    int32_t serial_send = 0;    // serial approach: the update of iteration k is sent when Compute(k) ends, not on entering k
     int32_t stale_reuse = 0;    // 1: a usable update an earlier Recv already returned is reduced again (HOP_STALE_REUSE)
     std::vector<int32_t> b;
 };

@@ -15,6 +15,8 @@
 //     available from every out-neighbour" is Iter(j) >= Iter(i) + 1 - max_ig for all of them, and
 //     the straggler test of Section 5 (how many tokens the out-neighbours hold for me) is
 //     min_j Iter(j) - Iter(i) - 1 iterations behind the slowest out-neighbour.
+// In the serial approach of Section 3.2 (Compute, Apply, Send, Recv, Reduce) an iteration's update leaves when its
+// Compute ends instead of when the iteration is entered; tokens move as before.
 // Time is integer ticks; only Compute takes time.  Transitions that fall on the same tick are
 // resolved in rounds: every worker whose inputs changed in the previous round decides from the
 // state that round left, then all decisions are committed.
@@ -46,7 +48,7 @@ struct Sim {
     std::vector<Phase> phase;
     std::vector<int32_t> jump_to;
     std::vector<int32_t> applied;                   // newest iteration whose Reduce/Apply is done (-1: none)
-    std::vector<std::vector<int32_t>> entered;      // iterations a worker has entered, ascending
+    std::vector<std::vector<int32_t>> entered;      // iterations whose update a worker has sent, ascending
     std::vector<std::vector<int64_t>> entered_seq;  // global order of those Send events (arrival order at every receiver)
     std::vector<int32_t> reduced;                   // per in-edge: newest version the receiver's completed Recvs have seen
     int64_t send_seq = 0;
@@ -67,10 +69,14 @@ struct Sim {
         return it == e.begin() ? -1 : *(it - 1);
     }
 
-    void enter(int32_t i, int32_t k) {
-        iter[i] = k;
+    void send(int32_t i, int32_t k) {
         entered[i].push_back(k);
         entered_seq[i].push_back(send_seq++);
+    }
+
+    void enter(int32_t i, int32_t k) {
+        iter[i] = k;
+        if (!p.serial_send) send(i, k);
         phase[i] = COMPUTE;
         compute_end.push({now + ticks[(size_t)i * iters + k], i});
     }
@@ -200,6 +206,7 @@ struct Sim {
                 compute_end.pop();
                 phase[i] = WAIT_RECV;
                 dirty[i] = 1;
+                if (p.serial_send) { send(i, iter[i]); touch_neighbours(i, dirty); }
             }
             for (;;) {
                 acts.clear();

@@ -63,20 +63,24 @@ def test_theorem1_bound_is_reached_on_a_chain():
 
 
 # ------------------------------------------------------------------ closed form (max-plus recurrence)
-def recurrence(n_in, T, iters, s, max_ig):
+def recurrence(n_in, T, iters, s, max_ig, serial=False):
     """start/finish times for b = 0, no skipping: a worker finishes Recv(k) once its compute is over
-    and every in-neighbour has entered iteration k - s; it enters k+1 once every out-neighbour has
-    entered k + 1 - max_ig."""
+    and every in-neighbour has sent iteration k - s -- on entering it (parallel approach) or at the end
+    of its Compute (serial approach, Section 3.2); it enters k+1 once every out-neighbour has entered
+    k + 1 - max_ig.  Returns (start, finish, sent)."""
     N = len(n_in)
     n_out = [[i for i in range(N) if j in n_in[i] and i != j] for j in range(N)]
     start = np.zeros((N, iters + 1), np.int64)
     fin = np.zeros((N, iters), np.int64)
+    sent = np.zeros((N, iters), np.int64)
     for k in range(iters):
+        for i in range(N):
+            sent[i, k] = start[i, k] + (int(T[i][k]) if serial else 0)
         for i in range(N):
             f = start[i, k] + int(T[i][k])
             for j in n_in[i]:
                 if j != i:
-                    f = max(f, start[j, max(k - s, 0)])
+                    f = max(f, sent[j, max(k - s, 0)])
             fin[i, k] = f
         for i in range(N):
             st = fin[i, k]
@@ -84,11 +88,12 @@ def recurrence(n_in, T, iters, s, max_ig):
                 for j in n_out[i]:
                     st = max(st, start[j, k + 1 - max_ig])
             start[i, k + 1] = st
-    return start, fin
+    return start, fin, sent
 
 
+@pytest.mark.parametrize("serial", [False, True])
 @pytest.mark.parametrize("s,max_ig", [(0, None), (0, 1), (0, 3), (2, None), (2, 2), (3, 1)])
-def test_times_and_versions_match_maxplus_recurrence(s, max_ig):
+def test_times_and_versions_match_maxplus_recurrence(s, max_ig, serial):
     rng = np.random.default_rng(7 + s)
     for name, n_in in GRAPHS:
         N = len(n_in)
@@ -101,27 +106,47 @@ def test_times_and_versions_match_maxplus_recurrence(s, max_ig):
         def chk(p):
             for i in range(N):
                 starts.setdefault((i, p.Iter[i]), p.now)
-        tr = op.simulate(n_in, T, iters, s=s, b=0, max_ig=max_ig, weight_mode=op.STALE_LINEAR, on_round=chk)
-        # every wait looks at a lower or equal level whose start time is already final, so one
-        # sweep per level evaluates the recurrence
-        st, fin = recurrence(n_in, T, iters, s, max_ig)
+        tr = op.simulate(n_in, T, iters, s=s, b=0, max_ig=max_ig, weight_mode=op.STALE_LINEAR, on_round=chk,
+                         stale_reduce=op.REUSE, serial=serial)
+        # in the parallel approach every wait looks at a lower or equal level whose start time is already final; in
+        # the serial approach the level's own send times only need its start times: one sweep per level either way
+        st, fin, sent = recurrence(n_in, T, iters, s, max_ig, serial)
         for i in range(N):
             for k in range(1, iters):
                 assert starts[(i, k)] == st[i, k], (name, i, k)
         assert tr.makespan == fin[:, iters - 1].max()
-        # generic position: consumed version = newest v <= k with start(j, v) <= finish(i, k)
+        # generic position: consumed version = newest v <= k sent before Recv(k) finished
         for i in range(N):
             for k in range(iters):
+                assert sorted(j for j, _, _ in tr.rec[(k, i)]) == sorted(n_in[i])
                 for (j, v, w) in tr.rec[(k, i)]:
                     if j == i:
                         assert v == k
                         continue
-                    cand = [u for u in range(0, k + 1) if st[j, u] < fin[i, k]]
-                    ties = [u for u in range(0, k + 1) if st[j, u] == fin[i, k]]
+                    cand = [u for u in range(0, k + 1) if sent[j, u] < fin[i, k]]
+                    ties = [u for u in range(0, k + 1) if sent[j, u] == fin[i, k]]
                     if not ties:
                         assert v == max(cand), (name, i, k, j)
                     assert k - s <= v <= k
                     assert w == v - (k - s) + 1
+
+
+def test_serial_approach_with_s0_waits_for_the_neighbours_compute():
+    """Section 3.2: in the serial approach the update of iteration k leaves after Compute(k), so with s = 0 a worker's
+    Recv(k) ends with the slowest in-neighbour's Compute(k); in the parallel approach that update was sent on entering k,
+    and only the worker's own Compute counts."""
+    n_in = [[0, 1], [1]]                                    # worker 0 listens to worker 1
+    T = np.array([[1, 1, 1], [5, 5, 5]], np.uint64)
+    par = op.simulate(n_in, T, 3, s=0, max_ig=None)
+    ser = op.simulate(n_in, T, 3, s=0, max_ig=None, serial=True)
+    assert (par.makespan, ser.makespan) == (15, 15)         # worker 1 alone sets the makespan
+    done = {}
+
+    def chk(p):
+        done.setdefault((p.serial, p.Iter[0]), p.now)
+    op.simulate(n_in, T, 3, s=0, max_ig=None, on_round=chk)
+    op.simulate(n_in, T, 3, s=0, max_ig=None, serial=True, on_round=chk)
+    assert done[(False, 1)] == 1 and done[(True, 1)] == 5   # tick at which worker 0 enters iteration 1
 
 
 # ------------------------------------------------------------------ tokens

@@ -11,7 +11,7 @@ from paper_1902_01064_b200 import hop, inputs
 KEYS = ("op", "ptr", "nbr", "ver", "num", "den")
 
 
-def both(n_in, ticks, iters, s, b, max_ig, max_skip, mode, exact=False, notify_ack=False, reduce=op.NEW_ONLY):
+def both(n_in, ticks, iters, s, b, max_ig, max_skip, mode, exact=False, notify_ack=False, reduce=op.NEW_ONLY, serial=False):
     ptr, idx = inputs.graph_to_csr(n_in)
     n_in = inputs.csr_to_lists(ptr, idx)                 # records list neighbours in ascending id order
     h = hop.Hop(ptr, idx, len(n_in), 8, s, b, max_skip)
@@ -21,9 +21,10 @@ def both(n_in, ticks, iters, s, b, max_ig, max_skip, mode, exact=False, notify_a
     h.set_option(hop.OPT_NOTIFY_ACK, 1 if notify_ack else 0)
     assert (hop.STALE_NEW_ONLY, hop.STALE_REUSE) == (op.NEW_ONLY, op.REUSE)
     h.set_option(hop.OPT_STALE_REDUCE, reduce)
+    h.set_option(hop.OPT_APPROACH, hop.APPROACH_SERIAL if serial else hop.APPROACH_PARALLEL)
     got = h.sim_run(ticks, iters).to_arrays()
     want_tr = op.simulate(n_in, ticks, iters, s, b, None if notify_ack else max_ig, max_skip, mode, backup_exact=exact,
-                          notify_ack=notify_ack, stale_reduce=reduce)
+                          notify_ack=notify_ack, stale_reduce=reduce, serial=serial)
     want = want_tr.to_arrays()
     h.close()
     return got, want, want_tr.makespan
@@ -195,3 +196,43 @@ def test_notify_ack_bit_exact():
         for flat in itertools.product((1, 2, 3), repeat=9):
             got, want, mk = both(n_in, np.asarray(flat, np.uint64).reshape(3, 3), 3, 0, 0, 1, 0, op.UNIFORM, notify_ack=True)
             assert_same(got, want, mk, (name, flat))
+
+
+def test_serial_approach_bit_exact():
+    """Serial approach (Section 3.2): updates leave at the end of Compute.  Random graphs with ties, stragglers, backup
+    workers, both Reduce sets, EXACT backup and skipping; plus an exhaustive sweep on the small graphs."""
+    rng = np.random.default_rng(314)
+    differs = 0
+    for trial in range(40):
+        N = int(rng.integers(3, 11))
+        n_in = [{i, (i - 1) % N} for i in range(N)]
+        for _ in range(int(rng.integers(0, 3 * N))):
+            a, c = rng.integers(0, N, 2)
+            n_in[int(a)].add(int(c))
+        n_in = [sorted(x) for x in n_in]
+        s = int(rng.integers(0, 4))
+        b = int(rng.integers(0, min(len(x) for x in n_in)))
+        max_skip = int(rng.integers(0, s + 2)) if trial % 2 else 0
+        max_ig = int(rng.integers(1, 5))
+        ticks = rng.choice([1, 1, 2, 5], size=(N, 20)).astype(np.uint64)
+        kw = dict(exact=bool(trial % 3 == 0), reduce=op.REUSE if trial % 4 == 0 else op.NEW_ONLY)
+        try:
+            got, want, mk = both(n_in, ticks, 20, s, b, max_ig, max_skip, op.STALE_LINEAR, serial=True, **kw)
+        except op.Deadlock:
+            continue
+        assert_same(got, want, mk, trial)
+        try:
+            par = both(n_in, ticks, 20, s, b, max_ig, max_skip, op.STALE_LINEAR, **kw)[0]
+            differs += par["makespan"] != got["makespan"] or not np.array_equal(par["ver"], got["ver"])
+        except op.Deadlock:
+            pass
+    assert differs > 10
+    for name, n_in in inputs.small_cases():
+        N = len(n_in)
+        for flat in itertools.product((1, 2), repeat=N * 2):
+            ticks = np.asarray(flat, np.uint64).reshape(N, 2)
+            for (s, b, max_skip) in [(0, 0, 0), (1, 0, 0), (1, 1, 0), (2, 0, 2), (1, 1, 1)]:
+                if any(b >= len(nb) for nb in n_in):
+                    continue
+                got, want, mk = both(n_in, ticks, 2, s, b, max(1, s), max_skip, op.STALE_LINEAR, serial=True)
+                assert_same(got, want, mk, (name, flat, s, b, max_skip))
