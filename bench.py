@@ -33,7 +33,20 @@ PROBE = 1024
 # capture at a smaller parameter count P (same trace; traffic grows in proportion to the columns).  bench_config sums
 # it over exactly the levels the timed region ran and scales by columns.  An entry is removed whenever its kernel, the
 # trace or the gradient kernel in front of it changes.
-NCU_LEVEL_TRAFFIC = {}
+NCU_LEVEL_TRAFFIC = {
+    # mix_bulk_kernel, configuration 4 at P = 1 280 000 (1.6 GB ring), levels 0..49
+    4: {"P": 1_280_000, "stale_reduce": 0, "bytes": [
+        949631744, 946553600, 1014903808, 1051767296, 1077729536, 1098407680, 1109040384, 1187247872, 1192221952, 1197970688,
+        1191731456, 1107171072, 1139162112, 1144458496, 1160219392, 1278473984, 1178610944, 1147541760, 1132332544, 1169202944,
+        1125859328, 1136917248, 1142645504, 1163851264, 1142777344, 1184135424, 1157984256, 1210966784, 1137357568, 1126909952,
+        1126151680, 1126361088, 1126566912, 1142518016, 1127042048, 1126310400, 1126188800, 1126434304, 1127273984, 1126737408,
+        1147016704, 1126343680, 1142218752, 1142830848, 1126672640, 1126331392, 1183859456, 1179703296, 1153357824, 1137044224]},
+    # mix_dense_tc_kernel, configuration 5 at P = 1 024 000 (1.0 GB ring), levels 0..29
+    5: {"P": 1_024_000, "stale_reduce": 0, "bytes": [
+        1532526848, 1530028288, 1579470592, 1534755328, 1534438144, 1534676992, 1534232064, 1534825472, 1542433792, 1546918912,
+        1538204416, 1542948352, 1571140352, 1551143936, 1542484480, 1547291648, 1554810880, 1543000320, 1542492160, 1535121152,
+        1534205696, 1539237632, 1534291200, 1538695424, 1542948096, 1542900992, 1554481408, 1559620864, 1534096384, 1534786816]},
+}
 
 
 def shard_columns(P: int, n: int, r: int, unit: int = 128):

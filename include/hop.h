@@ -237,9 +237,19 @@ int hop_step_host(hop_ctx* ctx, const int32_t* op, const int64_t* ptr, const int
                   const int32_t* ver, const int32_t* num, const int32_t* den,
                   float* probe_dst, int64_t probe_len);
 
-/* Synchronises and returns the device-side error word (0 = no kernel check failed; otherwise
- * a code in the top byte and a detail in the rest). */
+/* Synchronises and returns the device-side error word.  Every wait inside the kernels (on a copy, on a free
+ * stage, on the tensor pipeline) is bounded; a kernel that gives up records the first such event and returns, so
+ * the context and the GPU stay usable.  0 = nothing happened (HOP_OK); otherwise HOP_E_DEVICE, the word has a code
+ * in its top byte (1: mix_bulk_kernel, a tile's copies did not arrive; 2: mix_bulk_kernel, no stage became free;
+ * 3: mix_dense_tc_kernel, a pipeline wait ran out) and a detail in the low 24 bits (tile index or wait site), and
+ * hop_last_error names it.  The parameters written by that level are then undefined.  The word is sticky until
+ * hop_clear_status. */
 int hop_read_status(hop_ctx* ctx, int32_t* device_error_word);
+/* Resets the device-side error word (asynchronous on the bound stream). */
+int hop_clear_status(hop_ctx* ctx);
+/* Self-test of that mechanism: launches one warp that waits on a barrier nothing completes, gives up after `polls`
+ * polls (1..65536, ~32 ns apart) and records code 1 with `detail`.  hop_read_status then reports HOP_E_DEVICE. */
+int hop_selftest_bounded_wait(hop_ctx* ctx, int32_t polls, int32_t detail);
 
 /* out[10] (host) for a level of the loaded trace: distinct consumed slices U_k, NORMAL records,
  * JUMP records, consumed entries sum_i |C_{i,k}|, tile width chosen, kernel chosen (hop_mix_kernel),

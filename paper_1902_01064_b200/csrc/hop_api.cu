@@ -792,7 +792,30 @@ extern "C" int hop_read_status(hop_ctx* c, int32_t* word) {
     if (!c->d_err) return HOP_OK;
     HOP_CUDA(c, cudaStreamSynchronize(c->stream));
     HOP_CUDA(c, cudaMemcpy(word, c->d_err, sizeof(int32_t), cudaMemcpyDeviceToHost));
-    if (*word != 0) HOP_FAIL(c, HOP_E_DEVICE, "a kernel gave up waiting (status word " + std::to_string(*word) + ")");
+    if (*word != 0) {
+        static const char* what[] = {"unknown", "mix_bulk_kernel: a tile's copies did not arrive", "mix_bulk_kernel: no stage became free",
+                                     "mix_dense_tc_kernel: a pipeline wait ran out"};
+        const int code = (*word >> 24) & 0xff;
+        HOP_FAIL(c, HOP_E_DEVICE, std::string("a kernel gave up waiting -- ") + what[code >= 1 && code <= 3 ? code : 0] +
+                                  " (status word " + std::to_string(*word) + ", detail " + std::to_string(*word & 0xffffff) + ")");
+    }
+    return HOP_OK;
+}
+
+extern "C" int hop_clear_status(hop_ctx* c) {
+    if (!c) return HOP_E_ARG;
+    if (!c->d_err) return HOP_OK;
+    HOP_CUDA(c, cudaMemsetAsync(c->d_err, 0, sizeof(int32_t), c->stream));
+    return HOP_OK;
+}
+
+extern "C" int hop_selftest_bounded_wait(hop_ctx* c, int32_t polls, int32_t detail) {
+    if (!c) return HOP_E_ARG;
+    if (polls < 1 || polls > 65536) HOP_FAIL(c, HOP_E_ARG, "hop_selftest_bounded_wait: polls must be in [1, 65536]");
+    if (!c->bound) HOP_FAIL(c, HOP_E_STATE, "hop_selftest_bounded_wait: bind buffers first");
+    const int e = hop_launch_wait_selftest(c->d_err, (uint32_t)polls, detail, c->stream);
+    if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("self-test launch: ") + cudaGetErrorString((cudaError_t)e));
+    c->launches += 1;
     return HOP_OK;
 }
 

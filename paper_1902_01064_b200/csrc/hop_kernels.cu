@@ -231,6 +231,24 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 __device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Self-test of the bounded wait: one warp waits on a barrier that nothing will ever complete, gives up after `polls`
+// polls, records ERR_FULL_WAIT with `detail` and returns -- the path a lost copy would take in mix_bulk_kernel.
+__global__ void __launch_bounds__(32)
+wait_selftest_kernel(int32_t* __restrict__ err_word, uint32_t polls, int32_t detail) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    bool done = false;
+    for (uint32_t it = 0; it < polls && !done; ++it) {
+        done = mbar_try_wait(&bar, 0);
+        if (!done) __nanosleep(32);
+    }
+    if (!done && threadIdx.x == 0) atomicCAS(err_word, 0, ERR_FULL_WAIT | (detail & 0xffffff));
+}
+
 // A record as the bulk kernel keeps it in shared memory: everything that does not depend on the tile is worked out
 // once per block (the generic record costs ~60 instructions per tile and record in address arithmetic and flags).
 struct alignas(16) BulkRec {
@@ -600,17 +618,19 @@ svm_dense_grad_kernel(float* __restrict__ G, int64_t P, HopLevelDev lv, const fl
 // Margins, coefficients and gradient of one worker's minibatch in one block (small problems: the three steps as separate
 // launches cost more in launch latency than in work).  Same arithmetic in the same order as svm_margin_dense_kernel
 // followed by svm_dense_grad_kernel: a warp per row for the margins, a thread per column for the gradient.
-constexpr int kFusedSvmThreads = 256;
+// The kernel is latency-bound (a few KB per worker): up to 32 warps take one minibatch row each, so all margins cost
+// one round of loads, and a gradient thread keeps 32 rows in flight.
+constexpr int kFusedSvmThreads = 1024;
 __global__ void __launch_bounds__(kFusedSvmThreads)
 svm_dense_fused_kernel(const float* __restrict__ X, float* __restrict__ G, int64_t P, int S, HopLevelDev lv,
                        const float* __restrict__ A, const float* __restrict__ y, int R, int B, int loss) {
     extern __shared__ float s_coef[];      // [B]
     launch_dependents();
     const int worker = lv.grad_workers[blockIdx.x];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
     const int64_t row0 = (int64_t)worker * R + (int64_t)(lv.level % (R / B)) * B;
     const float* x = X + ((int64_t)worker * S + lv.level % S) * P;
-    for (int r = warp; r < B; r += kFusedSvmThreads / 32) {
+    for (int r = warp; r < B; r += warps) {
         const float* arow = A + (row0 + r) * P;
         double m = 0.0;
         for (int64_t p = lane; p < P; p += 32) m += (double)arow[p] * (double)x[p];
@@ -618,10 +638,17 @@ svm_dense_fused_kernel(const float* __restrict__ X, float* __restrict__ G, int64
         if (lane == 0) s_coef[r] = loss_coefficient(y[row0 + r], m, B, loss);
     }
     __syncthreads();
-    for (int64_t p = threadIdx.x; p < P; p += kFusedSvmThreads) {
+    for (int64_t p = threadIdx.x; p < P; p += blockDim.x) {
         const float* a0 = A + row0 * P + p;
         float g = 0.f;
         int r = 0;
+        for (; r + 32 <= B; r += 32) {        // the loads first, then the multiply-adds in row order
+            float a[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) a[i] = a0[(int64_t)(r + i) * P];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) g = fmaf(s_coef[r + i], a[i], g);
+        }
         for (; r + 8 <= B; r += 8) {
             float a[8];
 #pragma unroll
@@ -775,7 +802,8 @@ int hop_launch_svm_dense(const HopLaunchCfg& c, const HopLevelDev& lv, const flo
     const int warps = lv.nG * B;
     cudaStream_t st = (cudaStream_t)c.stream;
     if (phase == 0 && hop_svm_dense_is_fused(c.P, B)) {
-        svm_dense_fused_kernel<<<lv.nG, kFusedSvmThreads, (size_t)B * sizeof(float), st>>>(c.X, c.G, c.P, c.s + 1, lv, A, y, R, B, c.loss);
+        const int threads = std::min(kFusedSvmThreads, std::max(128, std::max(32 * B, (int)((c.P + 31) / 32 * 32))));
+        svm_dense_fused_kernel<<<lv.nG, threads, (size_t)B * sizeof(float), st>>>(c.X, c.G, c.P, c.s + 1, lv, A, y, R, B, c.loss);
         return (int)cudaGetLastError();
     }
     if (phase != 2)
@@ -808,6 +836,11 @@ int hop_launch_svm_csr_apply(const HopLaunchCfg& c, const HopLevelDev& lv, const
     if (lv.nG == 0) return 0;
     const int warps = lv.nG * B;
     svm_csr_apply_kernel<<<(warps * 32 + 255) / 256, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.P, c.s + 1, c.lr, lv, row_ptr, col, val, R, B, coef, slot_shift);
+    return (int)cudaGetLastError();
+}
+
+int hop_launch_wait_selftest(int32_t* err_word, uint32_t polls, int32_t detail, void* stream) {
+    wait_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(err_word, polls, detail);
     return (int)cudaGetLastError();
 }
 

@@ -56,6 +56,8 @@ SIGNATURES = {
     "hop_step_end": [_p],
     "hop_step_host": [_p, _p, _p, _p, _p, _p, _p, _p, _i64],
     "hop_read_status": [_p, C.POINTER(_i32)],
+    "hop_clear_status": [_p],
+    "hop_selftest_bounded_wait": [_p, _i32, _i32],
     "hop_level_stats": [_p, _i32, _p],
     "hop_timing_enable": [_p, _i32],
     "hop_timing_read": [_p, _p, _p, C.POINTER(_i64)],
@@ -217,6 +219,18 @@ class Hop:
         w = _i32()
         self._chk(lib.hop_read_status(self.h, C.byref(w)))
         return w.value
+
+    def read_status_word(self):
+        """(return code, status word) without raising: HOP_E_DEVICE and the word a kernel left when it gave up a wait."""
+        w = _i32()
+        rc = lib.hop_read_status(self.h, C.byref(w))
+        return rc, w.value
+
+    def clear_status(self):
+        self._chk(lib.hop_clear_status(self.h))
+
+    def selftest_bounded_wait(self, polls=256, detail=0):
+        self._chk(lib.hop_selftest_bounded_wait(self.h, polls, detail))
 
     def level_stats(self, level):
         out = np.zeros(10, np.int64)

@@ -688,3 +688,25 @@ def test_svm_rebind_between_graph_replays_uses_the_new_buffers(cfg, P, iters):
         scale = np.abs(ref[i]).max() + 1e-30
         assert np.abs(got[i] - ref[i]).max() <= 1e-5 * scale
     g.h.close()
+
+
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
+    # a bounded wait that nothing satisfies returns by itself; the host sees HOP_E_DEVICE with the code and the detail
+    w = workload(3, P=1024, iters=6)
+    g = GpuRun(w)
+    ref = GpuRun(w).run(w.iters)
+    assert g.h.read_status_word() == (hop.OK, 0)
+    g.h.selftest_bounded_wait(polls=200, detail=4242)
+    rc, word = g.h.read_status_word()
+    assert rc == hop.E_DEVICE and word >> 24 == 1 and word & 0xffffff == 4242
+    with pytest.raises(hop.HopError) as e:
+        g.h.read_status()
+    assert e.value.code == hop.E_DEVICE and "copies did not arrive" in str(e.value) and "4242" in str(e.value)
+    g.h.selftest_bounded_wait(polls=50, detail=7)              # the first event is the one that is kept
+    assert g.h.read_status_word()[1] & 0xffffff == 4242
+    g.h.clear_status()
+    assert g.h.read_status_word() == (hop.OK, 0)
+    got = g.run(w.iters)                                       # the context and the device are still good
+    for i in range(w.N):
+        assert np.array_equal(got[i], ref[i])
+    g.h.close()
