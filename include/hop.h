@@ -104,6 +104,10 @@ typedef enum hop_grad_mode {
     HOP_GRAD_SVM_CSR = 3     /* hinge-loss linear SVM, CSR rows (hop_bind_svm_csr)                 */
 } hop_grad_mode;
 
+/* AUTO: TENSOR for dense levels (>= 32 active workers consuming >= 32 updates each, N <= 128, P % 128 == 0, no
+ * momentum or weight decay), else BULK when P % 4 == 0, else STAGED.  With P % 4 != 0 the rows of X are not 16-byte
+ * aligned, only 4-byte copies are possible and a level takes 2-3 times as long as with BULK: pad P to a multiple of 4
+ * where speed matters.  hop_level_stats reports the kernel each level was planned with. */
 typedef enum hop_mix_kernel {
     HOP_MIX_AUTO = 0,
     HOP_MIX_STAGED = 1,      /* column tile staged in shared memory by cp.async, two stages; any P */

@@ -20,8 +20,8 @@ Readings taken where the paper is silent (listed once more in the design notes):
   R2' Which satisfactory updates enter the Reduce (stale_reduce).  NEW_ONLY, the default, is what
       the paper prints three times: Eq. 2 sums over the in-neighbours whose update received in
       iteration k is satisfactory, Fig. alg3's Recv appends an update only when the newest
-      iteration among what this call dequeued is inside the bound, and Section 4.4 reduces the
-      newly received updates.  An in-neighbour whose newest update was already taken out of the
+      iteration among what this call dequeued is inside the bound, and Section 4.4 reduces what
+      has arrived since the last Reduce.  An in-neighbour whose newest update was already taken out of the
       queue by an earlier Recv of this worker still counts for the blocking test but adds no
       term; the own update is new in every iteration.  REUSE adds such an update again, with the
       lower weight Eq. 2 gives its age (every satisfactory in-neighbour contributes at every

@@ -80,7 +80,7 @@ int hop_validate_level(const HopGraph& g, const HopSimParams& p, int32_t level, 
         if (o == HOP_OP_JUMP && !(newest[i] <= level && newest[i] >= level - p.s)) return fail(i, "JUMP but the held version is outside [k-s, k]");
         const int32_t d = g.in_ptr[i + 1] - g.in_ptr[i];
         // Fig. alg4's count is about usable updates; with s > 0 and HOP_STALE_NEW_ONLY the Reduce may hold fewer
-        // (only the newly received ones, Eq. 2), down to the own update alone
+        // (only those that arrived since the previous Recv, Eq. 2), down to the own update alone
         const bool may_be_fewer = p.s > 0 && !p.stale_reuse;
         if (!may_be_fewer && e - a < d - p.b[i]) return fail(i, "fewer than |N_in| - b consumed updates");
         if (e - a > d) return fail(i, "more consumed updates than in-neighbours");
@@ -105,7 +105,7 @@ int hop_validate_level(const HopGraph& g, const HopSimParams& p, int32_t level, 
                 int32_t& last = (*taken)[edge - g.in_idx.begin()];
                 if (v < last) return fail(i, "version " + std::to_string(v) + " of worker " + std::to_string(j) + " is older than one consumed before");
                 if (v == last && !p.stale_reuse)
-                    return fail(i, "version " + std::to_string(v) + " of worker " + std::to_string(j) + " was consumed before (HOP_STALE_NEW_ONLY reduces newly received updates only)");
+                    return fail(i, "version " + std::to_string(v) + " of worker " + std::to_string(j) + " was consumed before (HOP_STALE_NEW_ONLY reduces an update once)");
                 last = v;
             }
             if (num[t] <= 0) return fail(i, "non-positive weight numerator");

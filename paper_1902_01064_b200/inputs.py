@@ -193,7 +193,7 @@ class Workload:
     sigma: float = 1e-3
     svm: Optional[SvmData] = None
     p0_zero: bool = False
-    stale_reduce: int = 0                  # 0: only newly received updates are reduced (Eq. 2 as printed); 1: reuse
+    stale_reduce: int = 0                  # 0: only updates that arrived since the previous Recv are reduced (Eq. 2 as printed); 1: reuse
     _p0: Optional[np.ndarray] = field(default=None, repr=False)
 
     @property

@@ -1,6 +1,6 @@
 """Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element.
 
-The configurations run under both readings of the bounded-staleness Reduce set (only newly received updates, the
+The configurations run under both readings of the bounded-staleness Reduce set (only updates that arrived since the worker's previous Recv, the
 default, as Eq. 2 and Fig. alg3 print it; or every update still inside the bound): `reduce` below.
 
 Tolerances (float32 path against a float64 oracle): max|delta| <= 1e-6 * max|x| after one level,

@@ -517,3 +517,21 @@ def test_notify_ack_prose_example_and_no_room_for_backup_workers():
     top[:] = [0, 0, 0]
     op.simulate(n_in, ticks, 10, s=0, b=1, max_ig=4, on_round=chk)
     assert top == [0, 4, 4]
+
+
+def test_notify_ack_chain_reaches_both_bounds_of_table1_exactly():
+    # Section 3.3 / Table 1, row NOTIFY-ACK, on a chain 0 -> 1 -> 2 whose last worker never finishes its first Compute:
+    # worker 1 reduces iterations 0 and 1 (ACKs both to worker 0) but cannot enter iteration 2 without ACK(0) from
+    # worker 2; worker 0 enters 2 on ACK(0), 3 on ACK(1), and stops there: a sender exactly 2 ahead of its receiver,
+    # a receiver exactly 1 ahead of its sender.
+    n_in = [[0], [0, 1], [1, 2]]
+    ticks = np.ones((3, 8), np.uint64)
+    ticks[2, 0] = STUCK
+    top = [0, 0, 0]
+
+    def chk(p):
+        if p.now < STUCK:
+            for i in range(3):
+                top[i] = max(top[i], p.Iter[i])
+    op.simulate(n_in, ticks, 8, notify_ack=True, on_round=chk)
+    assert top == [3, 1, 0]
