@@ -128,6 +128,8 @@ struct HopLaunchCfg {
     int32_t n_ents;
     int32_t early_x;    // the mix launch may overlap the tail of the gradient kernel launched just before it (which writes
                         // neither X nor M): programmatic dependent launch
+    int32_t dependent;  // CSR SVM kernels: launch as a programmatic dependent of the kernel in front (the kernel waits before it
+                        // touches anything that kernel, or one before it, may still be writing)
     void* stream;
 };
 int hop_launch_mix_staged(const HopLaunchCfg& c, const HopLevelDev& lv);

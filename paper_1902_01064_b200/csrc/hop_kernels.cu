@@ -337,6 +337,7 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
     const int rows = lv.U + nG * (MOMENTUM ? 2 : 1);
     const int64_t stage_floats = (int64_t)rows * w;
     const int64_t tiles = (P + w - 1) / w;
+    launch_dependents();     // a kernel behind that was launched as a dependent (the sparse apply) may fetch its static data
     if (!early_x) dependency_wait();
     if (tid == 0) {
         for (int s = 0; s < kBulkStages; ++s) { mbar_init(&full[s], kProducerWarps); mbar_init(&empty[s], kConsumerWarps); }
@@ -539,19 +540,46 @@ __device__ __forceinline__ float loss_coefficient(float y, double m, int B, int 
     return (float)(-(double)y / ((double)B * (1.0 + exp((double)y * m))));
 }
 
+// When launched as a programmatic dependent of the previous level's last kernel, the row's column indices and values
+// (static data) are fetched before dependency_wait and the parameter gather comes after it; launch_dependents comes
+// after the wait too, so that the mix-update kernel behind cannot start before everything in front has finished.
+constexpr int kCsrPrefetch = 4;      // elements per lane held in registers: rows of up to 128 stored elements in one round
 __global__ void __launch_bounds__(256)
 svm_margin_csr_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelDev lv, const int64_t* __restrict__ row_ptr,
                       const int32_t* __restrict__ col, const float* __restrict__ val, const float* __restrict__ y,
                       int R, int B, int loss, float* __restrict__ coef, double* __restrict__ margins_out) {
-    launch_dependents();
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-    if (gw >= lv.nG * B) return;
-    const int a = gw / B, r = gw - a * B;
-    const int worker = lv.grad_workers[a];
-    const int64_t row = (int64_t)worker * R + (int64_t)(lv.level % (R / B)) * B + r;
+    const bool live = gw < lv.nG * B;
+    int worker = 0, r = 0;
+    int64_t row = 0, t0 = 0, t1 = 0;
+    int32_t pc[kCsrPrefetch];
+    float pv[kCsrPrefetch];
+    if (live) {
+        const int a = gw / B;
+        r = gw - a * B;
+        worker = lv.grad_workers[a];
+        row = (int64_t)worker * R + (int64_t)(lv.level % (R / B)) * B + r;
+        t0 = row_ptr[row] + lane;
+        t1 = row_ptr[row + 1];
+#pragma unroll
+        for (int q = 0; q < kCsrPrefetch; ++q) {
+            const int64_t t = t0 + 32 * q;
+            pc[q] = t < t1 ? col[t] : 0;
+            pv[q] = t < t1 ? val[t] : 0.f;
+        }
+    }
+    dependency_wait();
+    launch_dependents();
+    if (!live) return;
     const float* x = X + ((int64_t)worker * S + lv.level % S) * P;
     double m = 0.0;
-    for (int64_t t = row_ptr[row] + lane; t < row_ptr[row + 1]; t += 32) m += (double)val[t] * (double)x[col[t]];
+    float xv[kCsrPrefetch];
+#pragma unroll
+    for (int q = 0; q < kCsrPrefetch; ++q) xv[q] = (t0 + 32 * q < t1) ? x[pc[q]] : 0.f;     // the gathers in flight together
+#pragma unroll
+    for (int q = 0; q < kCsrPrefetch; ++q)
+        if (t0 + 32 * q < t1) m += (double)pv[q] * (double)xv[q];                           // a lane's elements in their order
+    for (int64_t t = t0 + 32 * kCsrPrefetch; t < t1; t += 32) m += (double)val[t] * (double)x[col[t]];
     m = warp_sum(m);
     if (lane == 0) {
         if (margins_out) margins_out[(int64_t)worker * B + r] = m;     // partial margin over this shard's columns
@@ -661,21 +689,43 @@ svm_dense_fused_kernel(const float* __restrict__ X, float* __restrict__ G, int64
     }
 }
 
-// Sparse Apply after the dense mix: x_{k+1,i}[col] -= lr * coef_r * val, one warp per row.
+// Sparse Apply after the dense mix: x_{k+1,i}[col] -= lr * coef_r * val, one warp per row.  As a programmatic dependent of
+// the mix-update kernel it fetches the row's static data first and touches the coefficients and X only after dependency_wait.
 __global__ void __launch_bounds__(256)
 svm_csr_apply_kernel(float* __restrict__ X, int64_t P, int S, float lr, HopLevelDev lv, const int64_t* __restrict__ row_ptr,
                      const int32_t* __restrict__ col, const float* __restrict__ val, int R, int B,
                      const float* __restrict__ coef, int slot_shift) {
+    launch_dependents();
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-    if (gw >= lv.nG * B) return;
-    const int a = gw / B, r = gw - a * B;
-    const int worker = lv.grad_workers[a];
+    const bool live = gw < lv.nG * B;
+    int worker = 0, r = 0;
+    int64_t t0 = 0, t1 = 0;
+    int32_t pc[kCsrPrefetch];
+    float pv[kCsrPrefetch];
+    if (live) {
+        const int a = gw / B;
+        r = gw - a * B;
+        worker = lv.grad_workers[a];
+        const int64_t row = (int64_t)worker * R + (int64_t)(lv.level % (R / B)) * B + r;
+        t0 = row_ptr[row] + lane;
+        t1 = row_ptr[row + 1];
+#pragma unroll
+        for (int q = 0; q < kCsrPrefetch; ++q) {
+            const int64_t t = t0 + 32 * q;
+            pc[q] = t < t1 ? col[t] : -1;
+            pv[q] = t < t1 ? val[t] : 0.f;
+        }
+    }
+    dependency_wait();
+    if (!live) return;
     const float cf = coef[(int64_t)worker * B + r];
     if (cf == 0.f) return;
-    const int64_t row = (int64_t)worker * R + (int64_t)(lv.level % (R / B)) * B + r;
     float* x = X + ((int64_t)worker * S + (lv.level + slot_shift) % S) * P;
     const float scale = -lr * cf;
-    for (int64_t t = row_ptr[row] + lane; t < row_ptr[row + 1]; t += 32) atomicAdd(x + col[t], scale * val[t]);
+#pragma unroll
+    for (int q = 0; q < kCsrPrefetch; ++q)
+        if (pc[q] >= 0) atomicAdd(x + pc[q], scale * pv[q]);
+    for (int64_t t = t0 + 32 * kCsrPrefetch; t < t1; t += 32) atomicAdd(x + col[t], scale * val[t]);
 }
 
 // Serial approach (Compute, Apply, then Send): x_k <- x_k - lr * d in place for the level's NORMAL workers, with
@@ -818,16 +868,32 @@ int hop_launch_svm_dense(const HopLaunchCfg& c, const HopLevelDev& lv, const flo
     return (int)cudaGetLastError();
 }
 
+// One launch with or without the programmatic-serialization attribute (see dependency_wait above).
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_maybe_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, bool dependent, Args... args) {
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = grid; lc.blockDim = block; lc.dynamicSmemBytes = 0; lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = dependent ? 1 : 0;
+    return cudaLaunchKernelEx(&lc, kernel, KArgs(args)...);
+}
+
 int hop_launch_svm_csr_coef(const HopLaunchCfg& c, const HopLevelDev& lv, const int64_t* row_ptr, const int32_t* col,
                             const float* val, const float* y, int32_t R, int32_t B, float* coef, double* margins, int phase) {
     if (lv.nG == 0) return 0;
     const int warps = lv.nG * B;
     cudaStream_t st = (cudaStream_t)c.stream;
-    if (phase != 2)
-        svm_margin_csr_kernel<<<(warps * 32 + 255) / 256, 256, 0, st>>>(c.X, c.P, c.s + 1, lv, row_ptr, col, val, y, R, B, c.loss, coef,
-                                                                        phase == 1 ? margins : nullptr);
-    else
+    if (phase != 2) {
+        const cudaError_t e = launch_maybe_dependent(svm_margin_csr_kernel, dim3((warps * 32 + 255) / 256), dim3(256), st, c.dependent != 0,
+                                                     (const float*)c.X, c.P, (int)(c.s + 1), lv, row_ptr, col, val, y, (int)R, (int)B,
+                                                     (int)c.loss, coef, phase == 1 ? margins : (double*)nullptr);
+        if (e != cudaSuccess) return (int)e;
+    } else {
         svm_coef_from_margins_kernel<<<(warps + 255) / 256, 256, 0, st>>>(margins, lv, y, R, B, c.loss, coef);
+    }
     return (int)cudaGetLastError();
 }
 
@@ -835,7 +901,10 @@ int hop_launch_svm_csr_apply(const HopLaunchCfg& c, const HopLevelDev& lv, const
                              const float* val, int32_t R, int32_t B, const float* coef, int32_t slot_shift) {
     if (lv.nG == 0) return 0;
     const int warps = lv.nG * B;
-    svm_csr_apply_kernel<<<(warps * 32 + 255) / 256, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.P, c.s + 1, c.lr, lv, row_ptr, col, val, R, B, coef, slot_shift);
+    const cudaError_t e = launch_maybe_dependent(svm_csr_apply_kernel, dim3((warps * 32 + 255) / 256), dim3(256), (cudaStream_t)c.stream,
+                                                 c.dependent != 0, c.X, c.P, (int)(c.s + 1), c.lr, lv, row_ptr, col, val, (int)R, (int)B,
+                                                 coef, (int)slot_shift);
+    if (e != cudaSuccess) return (int)e;
     return (int)cudaGetLastError();
 }
 

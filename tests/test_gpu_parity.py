@@ -710,3 +710,50 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
     for i in range(w.N):
         assert np.array_equal(got[i], ref[i])
     g.h.close()
+
+
+def test_level_with_only_jump_records_between_normal_levels():
+    # A level whose active workers all jump has no gradient kernel in front of its mix-update launch, so that launch
+    # must not start early; the levels around it do.  Hand-made trace (two workers, s = 1, every update inside the
+    # bound reduced), run step by step and as one replayed graph, against the oracle's update rules on the same trace.
+    P, N, s = 4096, 2, 1
+    ptr, idx = inputs.graph_to_csr(inputs.complete(2))
+    w = inputs.Workload(0, "jump-only-level", N, P, 4, s=s, b=0, max_skip=1, max_ig=1, lr=0.1, momentum=0.9,
+                        weight_mode=inputs.STALE_LINEAR, grad_mode=inputs.GRAD_SYNTHETIC, in_ptr=ptr, in_idx=idx,
+                        ticks=np.ones((N, 4), np.uint64), grad_seed=5, stale_reduce=op.REUSE)
+    w._p0 = np.random.default_rng(2).standard_normal(P).astype(np.float32)
+    NORMAL, JUMP = op.NORMAL, op.JUMP
+    ops = np.array([[NORMAL, NORMAL], [JUMP, JUMP], [NORMAL, NORMAL], [NORMAL, NORMAL]], np.int32)
+    recs = {(0, 0): [(0, 0), (1, 0)], (0, 1): [(0, 0), (1, 0)],
+            (1, 0): [(0, 1), (1, 0)], (1, 1): [(0, 0), (1, 1)],           # own current parameters + the other's last sent update
+            (2, 0): [(0, 2), (1, 2)], (2, 1): [(0, 2), (1, 2)],           # iteration 1 was skipped by both: nothing of it was sent
+            (3, 0): [(0, 3), (1, 2)], (3, 1): [(0, 3), (1, 3)]}
+    t_ptr, nbr, ver, num = [0], [], [], []
+    den = np.zeros((4, N), np.int32)
+    for k in range(4):
+        for i in range(N):
+            for (j, v) in recs[(k, i)]:
+                nbr.append(j); ver.append(v); num.append(v - (k - s) + 1 if not (ops[k, i] == JUMP and j == i) else s + 1)
+            den[k, i] = sum(num[t_ptr[-1]:])
+            t_ptr.append(len(nbr))
+    tr = dict(op=ops, ptr=np.asarray(t_ptr, np.int64), nbr=np.asarray(nbr, np.int32), ver=np.asarray(ver, np.int32),
+              num=np.asarray(num, np.int32), den=den)
+    x0 = np.stack([w.p0() + w.perturbation(i) for i in range(N)])
+    X, newest = up.run_updates(tr, N, w.lr, w.momentum, x0.astype(np.float64), up.GradSynthetic(w.grad_seed, w.sigma, np.arange(P)), s=s)
+    want = [X[(i, newest[i])] for i in range(N)]
+    scale = max(np.abs(x).max() for x in want)
+    side = torch.cuda.Stream()
+    for graph in (False, True):
+        with torch.cuda.stream(side):
+            g = GpuRun(w, x0=x0)
+            g.h.load_trace(hop.Trace.from_arrays(*[tr[k] for k in KEYS]))
+            assert [g.h.level_stats(k)["normal"] for k in range(4)] == [2, 0, 2, 2] and g.h.level_stats(1)["jump"] == 2
+            if graph:
+                g.h.run(4)
+            else:
+                for _ in range(4):
+                    g.h.step()
+            assert g.h.read_status() == 0
+            for i in range(N):
+                assert np.abs(g.h.read_params(i) - want[i]).max() <= TOL_RUN * scale
+            g.h.close()
