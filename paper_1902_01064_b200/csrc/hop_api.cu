@@ -501,7 +501,9 @@ static int ensure_tc_maps(hop_ctx* c) {
 
 // phase 0: the whole level.  phase 1: the gradient phase only (SVM modes stop after the partial margins).
 // phase 2: the rest (SVM modes start from the margins the caller has summed over the column shards).
-static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, const TcPtrs& tc, int phase = 0) {
+// chained: the operation in front of this level on the stream is the previous level of the same hop_run call (a kernel of
+// this library), not something the caller enqueued.
+static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, const TcPtrs& tc, int phase = 0, bool chained = false) {
     size_t t0 = 0, t1 = 0;
     HopLaunchCfg cfg{};
     cfg.X = c->X; cfg.M = c->M; cfg.G = c->G; cfg.P = c->P; cfg.N = c->g.N; cfg.s = c->s;
@@ -522,9 +524,10 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, c
             c->launches += (phase == 1 || (phase == 0 && hop_svm_dense_is_fused(c->P, c->svmB))) ? 1 : 2;
             grad_kernel_in_front = true; break;
         case HOP_GRAD_SVM_CSR:
-            // parallel approach, whole level in one call: the margin kernel is a programmatic dependent of the previous level's
-            // last kernel (it fetches its static row data while that kernel drains, then waits), and the mix-update of it
-            cfg.dependent = (phase == 0 && !c->serial) ? 1 : 0;
+            // parallel approach inside hop_run: the margin kernel is a programmatic dependent of the previous level's last
+            // kernel (it fetches its static row data while that kernel drains, then waits), and the mix-update of it.  Not
+            // for the first level of a call: what the caller enqueued in front may still be writing the row data.
+            cfg.dependent = (phase == 0 && !c->serial && chained) ? 1 : 0;
             e = hop_launch_svm_csr_coef(cfg, lv, c->svmRowPtr, c->svmCol, c->svmVal, c->svmY, c->svmR, c->svmB, c->coef, c->margins, phase);
             c->launches += 1; grad_kernel_in_front = true; break;
         default: break;
@@ -623,10 +626,10 @@ extern "C" int hop_step(hop_ctx* c) {
     return HOP_OK;
 }
 
-static int enqueue_level(hop_ctx* c, int32_t k) {
+static int enqueue_level(hop_ctx* c, int32_t k, bool chained) {
     const HopLevelHost& L = c->levels[k];
     HopLevelDev lv{c->d_i32 + L.off_src, c->d_rec + L.off_rec, c->d_ent + L.off_ent, c->d_i32 + L.off_gw, L.U, L.nA, L.nG, k};
-    return run_level(c, L, lv, TcPtrs{c->d_tcw + L.off_tcw, c->d_tcrows + L.off_tcrows, c->d_tcsrc + L.off_tcsrc});
+    return run_level(c, L, lv, TcPtrs{c->d_tcw + L.off_tcw, c->d_tcrows + L.off_tcrows, c->d_tcsrc + L.off_tcsrc}, 0, chained);
 }
 
 extern "C" int hop_run(hop_ctx* c, int32_t n_levels) {
@@ -643,14 +646,14 @@ extern "C" int hop_run(hop_ctx* c, int32_t n_levels) {
     const bool graph = c->use_graph && c->stream != nullptr && !c->timing && c->grad_mode != HOP_GRAD_EXTERNAL && n_levels > 1;
     if (!graph) {
         for (int32_t k = first; k < first + n_levels; ++k)
-            if ((rc = enqueue_level(c, k))) return rc;
+            if ((rc = enqueue_level(c, k, k > first))) return rc;
     } else {
         auto key = std::make_pair(first, n_levels);
         auto it = c->graphs.find(key);
         if (it == c->graphs.end()) {
             const int64_t launches_before = c->launches;
             HOP_CUDA(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeRelaxed));
-            for (int32_t k = first; k < first + n_levels && !rc; ++k) rc = enqueue_level(c, k);
+            for (int32_t k = first; k < first + n_levels && !rc; ++k) rc = enqueue_level(c, k, k > first);
             cudaGraph_t g = nullptr;
             const cudaError_t ce = cudaStreamEndCapture(c->stream, &g);
             const int64_t in_graph = c->launches - launches_before;

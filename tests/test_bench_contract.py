@@ -28,3 +28,24 @@ def test_other_ranks_of_the_reference_arm_do_no_work():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
                        capture_output=True, text=True, timeout=120, cwd=ROOT, env=env)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_ncu_traffic_tables_cover_every_level_of_their_workloads():
+    """roofline.traffic is summed over the levels the timed region ran: the per-level tables must have one value per level
+    of the configuration's trace, be plausible against the algorithmic bytes of that level, and name the trace they
+    were captured on."""
+    import numpy as np
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_1902_01064_b200 import hop, inputs
+    for cfg, cap in bench.NCU_LEVEL_TRAFFIC.items():
+        w = inputs.make_workload(cfg, P=cap["P"])
+        assert len(cap["bytes"]) == w.iters and cap["stale_reduce"] == w.stale_reduce
+        h = hop.from_workload(w)
+        t = h.sim_run(w.ticks, w.iters).to_arrays()
+        h.close()
+        for k in range(w.iters):
+            lo, hi = t["ptr"][k * w.N], t["ptr"][(k + 1) * w.N]
+            U = len(set(zip(t["nbr"][lo:hi].tolist(), t["ver"][lo:hi].tolist())))
+            alg = 4 * cap["P"] * (U + int((t["op"][k] == 1).sum()) + int((t["op"][k] != 0).sum()))
+            assert 0.9 < cap["bytes"][k] / alg < 1.05, (cfg, k, cap["bytes"][k] / alg)
