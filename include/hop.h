@@ -105,14 +105,14 @@ typedef enum hop_grad_mode {
 } hop_grad_mode;
 
 /* AUTO: TENSOR for dense levels (>= 32 active workers consuming >= 32 updates each, N <= 128, P % 128 == 0, no
- * momentum or weight decay), else BULK when P % 4 == 0, else STAGED.  With P % 4 != 0 the rows of X are not 16-byte
- * aligned, only 4-byte copies are possible and a level takes 2-3 times as long as with BULK: pad P to a multiple of 4
- * where speed matters.  hop_level_stats reports the kernel each level was planned with. */
+ * momentum or weight decay), else BULK (STAGED only when P % 4 != 0 and the level's tables exceed 32 KB of shared
+ * memory).  hop_level_stats reports the kernel each level was planned with. */
 typedef enum hop_mix_kernel {
     HOP_MIX_AUTO = 0,
     HOP_MIX_STAGED = 1,      /* column tile staged in shared memory by cp.async, two stages; any P */
     HOP_MIX_BULK = 2,        /* same, slices fetched by bulk copies, producer and consumer warps;  */
-                             /* needs P % 4 == 0 (AUTO picks it then, else STAGED)                 */
+                             /* any P (with P % 4 != 0 the rows are not 16-byte aligned: each is   */
+                             /* fetched from the boundary below it and read back with scalar loads) */
     HOP_MIX_TENSOR = 3       /* dense graphs: W_k * X on tcgen05 tensor cores, 3xTF32              */
 } hop_mix_kernel;
 

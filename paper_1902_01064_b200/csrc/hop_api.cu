@@ -364,14 +364,19 @@ static int plan_level(hop_ctx* c, HopLevelHost& L, bool allow_tensor = true) {
         L.alg_bytes = 4 * c->P * ((int64_t)L.U + nG + L.nA);
         return HOP_OK;
     }
-    if (kernel == HOP_MIX_AUTO || kernel == HOP_MIX_TENSOR) kernel = (c->P % 4 == 0) ? HOP_MIX_BULK : HOP_MIX_STAGED;
-    if (kernel == HOP_MIX_BULK && c->P % 4 != 0) HOP_FAIL(c, HOP_E_UNSUPPORTED, "the bulk-copy mix kernel needs P to be a multiple of 4");
     const int rows = std::max(1, L.stage_rows);
     const int64_t tb = ((int64_t)L.recs.size() * sizeof(HopRecord) + (int64_t)L.ents.size() * sizeof(HopEntry) + 127) / 128 * 128;
-    L.table_smem = (kernel == HOP_MIX_BULK && tb <= hop_mix_table_limit()) ? (int32_t)tb : 0;
+    const bool tables_fit = tb <= hop_mix_table_limit();
+    const bool unaligned = c->P % 4 != 0;
+    // The bulk-copy kernel takes any P; with P % 4 != 0 it needs its tables in shared memory and a staged row of w + 4 floats.
+    if (kernel == HOP_MIX_AUTO || kernel == HOP_MIX_TENSOR) kernel = (!unaligned || tables_fit) ? HOP_MIX_BULK : HOP_MIX_STAGED;
+    if (kernel == HOP_MIX_BULK && unaligned && !tables_fit)
+        HOP_FAIL(c, HOP_E_UNSUPPORTED, "the bulk-copy mix kernel with P not a multiple of 4 needs the level's tables to fit shared memory");
+    const bool padded = kernel == HOP_MIX_BULK && unaligned;
+    L.table_smem = (kernel == HOP_MIX_BULK && tables_fit) ? (int32_t)tb : 0;
     const int64_t budget = (hop_mix_smem_budget(kernel) - L.table_smem) / hop_mix_stages(kernel);
-    int64_t w = budget / ((int64_t)rows * 4);
-    const int unit = (c->P % 4 == 0) ? 4 : 1;
+    int64_t w = budget / ((int64_t)rows * 4) - (padded ? 4 : 0);
+    const int unit = (!unaligned || padded) ? 4 : 1;
     if (w >= 128) w = std::min<int64_t>(1024, w / 128 * 128);
     else if (w >= 32) w = w / 32 * 32;
     else w = w / unit * unit;
@@ -380,8 +385,12 @@ static int plan_level(hop_ctx* c, HopLevelHost& L, bool allow_tensor = true) {
     w = std::min<int64_t>(w, Pr);
     L.tile_w = (int32_t)w;
     L.kernel = kernel;
-    for (HopEntry& e : L.ents) e.u *= L.tile_w;     // slice index -> float offset of its row in a staged tile
-    for (HopRecord& r : L.recs) if (r.self_u >= 0) r.self_u *= L.tile_w;
+    // slice index -> float offset of the slice's element 0 in a staged tile (padded rows: stride w + 4, plus the distance of
+    // the row's first element from the 16-byte boundary below it, the same for every tile since w is a multiple of 4)
+    const int64_t stride = w + (padded ? 4 : 0);
+    auto offset_of = [&](int32_t slice) { return (int32_t)(slice * stride + (padded ? (((int64_t)L.src_row[slice] * c->P) & 3) : 0)); };
+    for (HopEntry& e : L.ents) e.u = offset_of(e.u);
+    for (HopRecord& r : L.recs) if (r.self_u >= 0) r.self_u = offset_of(r.self_u);
     // every distinct consumed slice once + gradient once + result once (+ momentum read and write)
     L.alg_bytes = 4 * c->P * ((int64_t)L.U + nG + L.nA + (mom ? 2 * (int64_t)nG : 0));
     return HOP_OK;

@@ -311,19 +311,57 @@ __device__ __forceinline__ void bulk_record(const BulkRec& r, const int4* __rest
     }
 }
 
+// The same for parameter counts that are not multiples of 4 (ALIGNED = false): a slice's staged copy starts at the 16-byte
+// boundary below its first element, so element c of the tile sits `shift` floats into its staged row (the shift is
+// folded into the table offsets) and is not 16-byte aligned in general: a lane takes every 32nd column with scalar
+// shared-memory loads (the same number of shared-memory wavefronts as the vector form, four times the load instructions)
+// and scalar, coalesced global stores.  Same multiply-adds in the same order.
+template <bool MOMENTUM, bool DECAY>
+__device__ __forceinline__ void bulk_record_scalar(const BulkRec& r, const int4* __restrict__ ents2, const float* __restrict__ stage,
+                                                   int ws, int wd, int nG, float lr, float mu, float lam, float* __restrict__ Xc,
+                                                   float* __restrict__ Mc, int64_t P, int lane) {
+#pragma unroll 1
+    for (int c = lane; c < wd; c += 32) {
+        float acc = 0.f;
+        const float* sc = stage + c;
+        const int4* e = ents2 + (r.ent_begin >> 1);
+#pragma unroll 1
+        for (int g = 0; g < r.groups; ++g, e += 2) {
+            const int4 e01 = e[0], e23 = e[1];
+            const float v0 = sc[e01.x], v1 = sc[e01.z], v2 = sc[e23.x], v3 = sc[e23.z];
+            acc = fmaf(__int_as_float(e01.y), v0, acc); acc = fmaf(__int_as_float(e01.w), v1, acc);
+            acc = fmaf(__int_as_float(e23.y), v2, acc); acc = fmaf(__int_as_float(e23.w), v3, acc);
+        }
+        if (DECAY && r.self_off >= 0 && r.g_off < 0) acc = fmaf(-lr * lam, sc[r.self_off], acc);
+        if (r.g_off >= 0) {
+            float g = sc[r.g_off];
+            if (DECAY && r.self_off >= 0) g = fmaf(lam, sc[r.self_off], g);
+            if constexpr (MOMENTUM) {
+                g = fmaf(mu, sc[r.g_off + nG * ws], g);
+                Mc[(int64_t)r.worker * P + c] = g;
+            }
+            acc = fmaf(-lr, g, acc);
+        }
+        Xc[r.out_off + c] = acc;
+    }
+}
+
 // mix_bulk: persistent blocks; the first kProducerWarps warps are producers (asynchronous bulk copies of
 // every staged row of the next tile, rows dealt round-robin to the producer lanes, completion counted
 // in bytes on an mbarrier), the other kConsumerWarps warps consume.  Two stages.
-// Requires P % 4 == 0 and 16-byte aligned base pointers (bulk copies move multiples of 16 bytes).
+// 16-byte aligned base pointers (bulk copies move multiples of 16 bytes from 16-byte boundaries).  ALIGNED: P % 4 == 0, every
+// row piece is such a copy.  !ALIGNED: any P; a row piece is fetched from the 16-byte boundary below its first element
+// into a staged row of w + 4 floats (never past the end of the buffer it lies in: the last one to three floats of a
+// buffer come by plain loads), consumers use bulk_record_scalar, early_x is not used, the tables must be in shared memory.
 // early_x != 0: the launch carries the programmatic-serialization attribute and the kernel in front of it in the stream
 // (the level's gradient kernel) writes neither X nor M: barrier set-up, the tables and the X / M rows of the first
 // kBulkStages tiles are then fetched while that kernel is still draining; the gradient rows and every store come
 // after dependency_wait.  early_x == 0: everything comes after it.
-template <bool MOMENTUM, bool DECAY>
+template <bool MOMENTUM, bool DECAY, bool ALIGNED = true>
 __global__ void __launch_bounds__(kBulkThreads, 1)
 mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __restrict__ G, int64_t P, int w,
                 int use_g, float lr, float mu, float lam, HopLevelDev lv, int table_bytes, int n_ents,
-                int32_t* __restrict__ err_word, int early_x) {
+                int32_t* __restrict__ err_word, int early_x, int ring_rows, int n_workers) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw);
     uint64_t* empty = full + kBulkStages;
@@ -335,10 +373,11 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nG = use_g ? lv.nG : 0;
     const int rows = lv.U + nG * (MOMENTUM ? 2 : 1);
-    const int64_t stage_floats = (int64_t)rows * w;
+    const int ws = ALIGNED ? w : w + 4;                    // floats per staged row
+    const int64_t stage_floats = (int64_t)rows * ws;
     const int64_t tiles = (P + w - 1) / w;
     launch_dependents();     // a kernel behind that was launched as a dependent (the sparse apply) may fetch its static data
-    if (!early_x) dependency_wait();
+    if (!(ALIGNED && early_x)) dependency_wait();
     if (tid == 0) {
         for (int s = 0; s < kBulkStages; ++s) { mbar_init(&full[s], kProducerWarps); mbar_init(&empty[s], kConsumerWarps); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -370,23 +409,50 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
         auto issue = [&](int64_t tile, int s, int which) {
             const int64_t c0 = tile * w;
             const int wd = (int)min((int64_t)w, P - c0);
-            const uint32_t bytes = (uint32_t)wd * 4u;
-            if (which != 2) {
-                if (lane == 0) mbar_expect_tx(&full[s], bytes * (uint32_t)my_rows);
-                __syncwarp();
-            }
             float* dst = stage0 + s * stage_floats;
-            auto wanted = [&](int r) { return which == 0 || ((r >= lv.U && r < lv.U + nG) == (which == 2)); };
+            if constexpr (ALIGNED) {
+                const uint32_t bytes = (uint32_t)wd * 4u;
+                if (which != 2) {
+                    if (lane == 0) mbar_expect_tx(&full[s], bytes * (uint32_t)my_rows);
+                    __syncwarp();
+                }
+                auto wanted = [&](int r) { return which == 0 || ((r >= lv.U && r < lv.U + nG) == (which == 2)); };
 #pragma unroll
-            for (int h = 0; h < kHoist; ++h) {
-                const int r = warp + (lane + 32 * h) * kProducerWarps;
-                if (src_h[h] && wanted(r)) bulk_g2s(dst + r * w, src_h[h] + c0, bytes, &full[s]);
+                for (int h = 0; h < kHoist; ++h) {
+                    const int r = warp + (lane + 32 * h) * kProducerWarps;
+                    if (src_h[h] && wanted(r)) bulk_g2s(dst + r * w, src_h[h] + c0, bytes, &full[s]);
+                }
+                for (int r = warp + (lane + 32 * kHoist) * kProducerWarps; r < rows; r += 32 * kProducerWarps)
+                    if (wanted(r)) bulk_g2s(dst + (int64_t)r * w, row_src(r) + c0, bytes, &full[s]);
+            } else {
+                // which is always 0 here.  A piece starts `a` floats above a 16-byte boundary: copy from that boundary, a
+                // whole number of 16-byte units; the staged row then holds the tile's element c at index a + c.
+                uint32_t mine = 0;
+                auto fetch = [&](int r, const float* rowbase) {
+                    const float* src = rowbase + c0;
+                    const uint32_t a = (uint32_t)((reinterpret_cast<uintptr_t>(src) >> 2) & 3u);
+                    const float* src0 = src - a;
+                    uint32_t n = (a + (uint32_t)wd + 3u) & ~3u;
+                    float* d = dst + (int64_t)r * ws;
+                    const float* end = r < lv.U ? X + (int64_t)ring_rows * P : (r < lv.U + nG ? G : M) + (int64_t)n_workers * P;
+                    if (src0 + n > end) {                       // last piece of the buffer: its last 1-3 floats by plain loads
+                        n -= 4;
+                        for (const float* q = src0 + n; q < end; ++q) d[q - src0] = *q;
+                    }
+                    if (n) { bulk_g2s(d, src0, n * 4u, &full[s]); mine += n * 4u; }
+                };
+#pragma unroll
+                for (int h = 0; h < kHoist; ++h)
+                    if (src_h[h]) fetch(warp + (lane + 32 * h) * kProducerWarps, src_h[h]);
+                for (int r = warp + (lane + 32 * kHoist) * kProducerWarps; r < rows; r += 32 * kProducerWarps) fetch(r, row_src(r));
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+                __syncwarp();                                   // the plain stores above are ordered before lane 0's arrival
+                if (lane == 0) mbar_expect_tx(&full[s], mine);  // bytes may complete before they are expected: the count is signed
             }
-            for (int r = warp + (lane + 32 * kHoist) * kProducerWarps; r < rows; r += 32 * kProducerWarps)
-                if (wanted(r)) bulk_g2s(dst + (int64_t)r * w, row_src(r) + c0, bytes, &full[s]);
         };
         int64_t tile = blockIdx.x;
-        if (early_x) {
+        if (ALIGNED && early_x) {
             // the first tiles' X and M rows while the gradient kernel may still be writing G (both stages are free)
             int pre = 0;
             for (int64_t t = tile; t < tiles && pre < kBulkStages; t += gridDim.x, ++pre) issue(t, pre, 1);
@@ -420,7 +486,7 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
                 b.out_off = (int64_t)r.out_row * P;
                 b.ent_begin = r.ent_begin;
                 b.groups = r.ent_count >> 2;
-                b.g_off = grad ? (lv.U + r.g_stage) * w : -1;
+                b.g_off = grad ? (lv.U + r.g_stage) * ws + (ALIGNED ? 0 : (int)(((int64_t)r.worker * P) & 3)) : -1;
                 b.self_off = (DECAY && r.g_stage >= 0 && r.self_u >= 0) ? r.self_u : -1;
                 b.worker = r.worker;
                 b.pad = 0;
@@ -431,7 +497,7 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
             for (int i = ct; i < n_ents; i += kConsumerThreads) sent[i] = ge[i];
             asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
         }
-        if (early_x) dependency_wait();      // no store before the kernel in front has finished (it may read the slot written here)
+        if (ALIGNED && early_x) dependency_wait();      // no store before the kernel in front has finished (it may read the slot written here)
         int64_t n = 0;
         for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++n) {
             const int s = (int)(n % kBulkStages);
@@ -442,9 +508,13 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
             const float* st = stage0 + s * stage_floats;
             if (table_bytes > 0) {
 #pragma unroll 1
-                for (int a = cw; a < lv.nA; a += kConsumerWarps)
-                    bulk_record<MOMENTUM, DECAY>(srec[a], sent2, st, w, wd, nG, lr, mu, lam, X + c0, MOMENTUM ? M + c0 : nullptr, P, lane);
-            } else {
+                for (int a = cw; a < lv.nA; a += kConsumerWarps) {
+                    if constexpr (ALIGNED)
+                        bulk_record<MOMENTUM, DECAY>(srec[a], sent2, st, w, wd, nG, lr, mu, lam, X + c0, MOMENTUM ? M + c0 : nullptr, P, lane);
+                    else
+                        bulk_record_scalar<MOMENTUM, DECAY>(srec[a], sent2, st, ws, wd, nG, lr, mu, lam, X + c0, MOMENTUM ? M + c0 : nullptr, P, lane);
+                }
+            } else if constexpr (ALIGNED) {
                 for (int a = cw; a < lv.nA; a += kConsumerWarps)
                     reduce_apply_record<4, MOMENTUM, DECAY>(lv.recs[a], lv.ents, st, w, wd, lv.U, nG, use_g != 0, lr, mu, lam, X, M, P, c0, lane);
             }
@@ -807,7 +877,9 @@ int hop_launch_mix_bulk(const HopLaunchCfg& c, const HopLevelDev& lv) {
     if (lv.nA == 0) return 0;
     const int nG = c.use_g ? lv.nG : 0;
     const int rows = lv.U + nG * (c.mu != 0.f ? 2 : 1);
-    const size_t smem = 128 + (size_t)c.table_smem + (size_t)kBulkStages * rows * c.tile_w * sizeof(float);
+    const bool aligned = c.P % 4 == 0;
+    if (!aligned && c.table_smem == 0) return (int)cudaErrorInvalidValue;      // the planner never asks for this
+    const size_t smem = 128 + (size_t)c.table_smem + (size_t)kBulkStages * rows * (c.tile_w + (aligned ? 0 : 4)) * sizeof(float);
     const int64_t tiles = (c.P + c.tile_w - 1) / c.tile_w;
     const int grid = (int)std::min<int64_t>(tiles, (int64_t)c.sm_count);
     cudaStream_t st = (cudaStream_t)c.stream;
@@ -818,19 +890,22 @@ int hop_launch_mix_bulk(const HopLaunchCfg& c, const HopLevelDev& lv) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
-    lc.numAttrs = c.early_x ? 1 : 0;
-#define HOP_LAUNCH_BULK(MO, DE)                                                                               \
+    const int early_x = (c.early_x && aligned) ? 1 : 0;
+    lc.numAttrs = early_x ? 1 : 0;
+#define HOP_LAUNCH_BULK(MO, DE, AL)                                                                           \
     do {                                                                                                      \
-        e = hop_allow_max_smem<mix_bulk_kernel<MO, DE>>();                                                    \
+        e = hop_allow_max_smem<mix_bulk_kernel<MO, DE, AL>>();                                                \
         if (e == cudaSuccess)                                                                                 \
-            e = cudaLaunchKernelEx(&lc, mix_bulk_kernel<MO, DE>, c.X, c.M, (const float*)c.G, c.P, (int)c.tile_w, (int)c.use_g, c.lr, c.mu, \
-                                   c.wd, lv, (int)c.table_smem, (int)c.n_ents, c.err_word, (int)c.early_x);  \
+            e = cudaLaunchKernelEx(&lc, mix_bulk_kernel<MO, DE, AL>, c.X, c.M, (const float*)c.G, c.P, (int)c.tile_w, (int)c.use_g, c.lr, c.mu, \
+                                   c.wd, lv, (int)c.table_smem, (int)c.n_ents, c.err_word, early_x, (int)(c.N * (c.s + 1)), (int)c.N); \
     } while (0)
+#define HOP_LAUNCH_BULK2(MO, DE) do { if (aligned) HOP_LAUNCH_BULK(MO, DE, true); else HOP_LAUNCH_BULK(MO, DE, false); } while (0)
     const bool mom = c.mu != 0.f, dec = c.wd != 0.f;
-    if (mom && dec) HOP_LAUNCH_BULK(true, true);
-    else if (mom) HOP_LAUNCH_BULK(true, false);
-    else if (dec) HOP_LAUNCH_BULK(false, true);
-    else HOP_LAUNCH_BULK(false, false);
+    if (mom && dec) HOP_LAUNCH_BULK2(true, true);
+    else if (mom) HOP_LAUNCH_BULK2(true, false);
+    else if (dec) HOP_LAUNCH_BULK2(false, true);
+    else HOP_LAUNCH_BULK2(false, false);
+#undef HOP_LAUNCH_BULK2
 #undef HOP_LAUNCH_BULK
     if (e != cudaSuccess) return (int)e;
     return (int)cudaGetLastError();

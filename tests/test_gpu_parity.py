@@ -141,8 +141,9 @@ def test_cfg2_full_size_whole_run():
 
 # ------------------------------------------------------------------ configuration 3: momentum + skipping
 @pytest.mark.parametrize("reduce", REDUCE)
-@pytest.mark.parametrize("kernel,P", [(hop.MIX_STAGED, 5000), (hop.MIX_BULK, 5000), (hop.MIX_STAGED, 4999),
-                                      (hop.MIX_BULK, 132), (hop.MIX_STAGED, 3)])
+@pytest.mark.parametrize("kernel,P", [(hop.MIX_STAGED, 5000), (hop.MIX_BULK, 5000), (hop.MIX_STAGED, 4999), (hop.MIX_BULK, 4999),
+                                      (hop.MIX_BULK, 132), (hop.MIX_STAGED, 3), (hop.MIX_BULK, 3), (hop.MIX_BULK, 4097),
+                                      (hop.MIX_BULK, 130), (hop.MIX_BULK, 1023)])
 def test_cfg3_reduced_full_run(kernel, P, reduce):
     w = workload(3, reduce, P=P)
     check(w, w.iters, TOL_RUN, kernel)
@@ -260,7 +261,7 @@ def test_external_gradients_and_tiny_shapes():
                             ticks=rng.integers(1, 9, size=(N, iters)).astype(np.uint64))
         w._p0 = rng.standard_normal(P).astype(np.float32)
         G = rng.standard_normal((iters, N, P)).astype(np.float32)
-        for kernel in ([hop.MIX_STAGED, hop.MIX_BULK] if P % 4 == 0 else [hop.MIX_STAGED]):
+        for kernel in (hop.MIX_STAGED, hop.MIX_BULK):          # the bulk-copy kernel takes any P (unaligned rows included)
             check(w, iters, TOL_RUN, kernel, perturb=True, external_G=G)
 
 
@@ -633,14 +634,19 @@ def test_options_set_after_load_trace_plan_the_levels_again():
     assert max(np.abs(got[i] - want[i]).max() for i in range(w.N)) <= TOL_RUN * scale
     # a value the loaded trace cannot be planned with is refused and leaves the context as it was
     g.h.close()
-    w = workload(3, P=4999, iters=6)
-    g = GpuRun(w, hop.MIX_STAGED)
-    with pytest.raises(hop.HopError) as e:
-        g.h.set_option(hop.OPT_MIX_KERNEL, hop.MIX_BULK)       # needs P % 4 == 0
-    assert e.value.code == hop.E_UNSUPPORTED
+    # a parameter count that is not a multiple of 4: the general kernel first, the bulk-copy kernel chosen after the load
+    w = workload(3, P=4999, iters=12)
+    x0 = np.stack([w.p0() + w.perturbation(i) for i in range(w.N)])
+    g = GpuRun(w, hop.MIX_STAGED, x0=x0)
     assert g.h.level_stats(1)["kernel"] == hop.MIX_STAGED
-    g.h.step()
-    assert g.h.read_status() == 0
+    g.h.set_option(hop.OPT_MIX_KERNEL, hop.MIX_BULK)
+    assert g.h.level_stats(1)["kernel"] == hop.MIX_BULK
+    got = g.run(w.iters)
+    want, scale = _oracle_state(w, x0, w.iters)
+    assert max(np.abs(got[i] - want[i]).max() for i in range(w.N)) <= TOL_RUN * scale
+    with pytest.raises(hop.HopError):
+        g.h.set_option(hop.OPT_MIX_KERNEL, 9)                  # refused; the context stays as it was
+    assert g.h.level_stats(1)["kernel"] == hop.MIX_BULK
     g.h.close()
 
 
@@ -757,3 +763,22 @@ def test_level_with_only_jump_records_between_normal_levels():
             for i in range(N):
                 assert np.abs(g.h.read_params(i) - want[i]).max() <= TOL_RUN * scale
             g.h.close()
+
+
+@pytest.mark.parametrize("P", [4999, 10001, 10002, 10003])
+def test_bulk_kernel_with_unaligned_rows_equals_the_general_kernel_bitwise(P):
+    # P % 4 = 3, 1, 2, 3: every row of the ring starts at a different distance from a 16-byte boundary; the last row of
+    # each buffer ends 1-3 floats short of one (the plain-load tail).  Same multiply-adds in the same order as the
+    # general kernel, so the results agree bit for bit; momentum, a jumping straggler and weight decay are on.
+    w = workload(3, P=P, iters=30)
+    x0 = np.stack([w.p0() + w.perturbation(i) for i in range(w.N)])
+    for variant in (None, dict(weight_decay=0.01)):
+        a = GpuRun(w, hop.MIX_STAGED, x0=x0, variant=variant)
+        b = GpuRun(w, hop.MIX_BULK, x0=x0, variant=variant)
+        assert a.h.level_stats(3)["kernel"] == hop.MIX_STAGED and b.h.level_stats(3)["kernel"] == hop.MIX_BULK
+        ra, rb = a.run(w.iters), b.run(w.iters)
+        for i in range(w.N):
+            assert np.array_equal(ra[i], rb[i])
+        assert torch.equal(a.M, b.M)
+        a.h.close()
+        b.h.close()
