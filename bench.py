@@ -117,6 +117,15 @@ class ClockSampler(threading.Thread):
                 "samples": len(self.samples)}
 
 
+def workload_config(cfg, w, P_global):
+    """The `config` object of the JSON line: what names the workload, the same for both arms of the benchmark."""
+    ring = w.N * (w.s + 1) * P_global * 4
+    return {"workload": f"config {cfg}: {w.name}", "N": w.N, "P": P_global, "s": w.s, "b": w.b, "levels": w.iters,
+            "stale_reduce": "new_only (Eq. 2 as printed)" if w.stale_reduce == 0 else "reuse",
+            "l2": ("inputs exceed L2 (ring %.1f GB over all GPUs): no flush between iterations" % (ring / 1e9)) if ring > 3e8
+                  else "ring fits L2: absolute numbers only"}
+
+
 def oracle_sample(w, budget_cols=131072, levels=6):
     """The CPU oracle, as it stands, on a bounded sample of the workload: the full protocol simulation
     plus `levels` levels of the fp64 update rules on `budget_cols` columns (the synthetic-gradient path
@@ -211,7 +220,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * (w.N / value), "higher_is_better": True, "scaling": "strong",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"config {args.config}: {w.name}", "N": w.N, "P": w.P, "s": w.s, "b": w.b, "levels": w.iters},
+            "config": workload_config(args.config, w, w.P),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -475,13 +484,11 @@ def bench_config(args, cfg, env):
             "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "value_mix_only": (normal_timed / mix_s) if mix_s > 0 else None,
-            "config": {"workload": f"config {cfg}: {w.name}", "N": w.N, "P": P_global, "P_per_gpu": w.P, "s": w.s, "b": w.b,
-                       "levels": w.iters, "trace_passes": steps / w.iters, "parallelism": f"column-sharded x{world}",
-                       "stale_reduce": "new_only (Eq. 2 as printed)" if w.stale_reduce == 0 else "reuse",
-                       "timed_levels": f"{timed_levels[0]}..{timed_levels[-1]}" if steps <= w.iters else f"whole trace x{steps / w.iters:.2f}",
-                       "l2": "inputs exceed L2 (ring %.1f GB per GPU)" % (ring_bytes / 1e9) if ring_bytes > 3e8 else "ring fits L2: absolute numbers only",
-                       "protocol_sim_ms": sim_ms,
-                       "launch": "hop_run: CUDA graph replay of the trace" if use_graph else "hop_step per level"},
+            "config": workload_config(cfg, w, P_global),
+            "run": {"P_per_gpu": w.P, "parallelism": f"column-sharded x{world}", "trace_passes": steps / w.iters,
+                    "timed_levels": f"{timed_levels[0]}..{timed_levels[-1]}" if steps <= w.iters else f"whole trace x{steps / w.iters:.2f}",
+                    "protocol_sim_ms": sim_ms,
+                    "launch": "hop_run: CUDA graph replay of the trace" if use_graph else "hop_step per level"},
             "roofline": roofline, "gpu_launches": int(launches), "clocks": sampler.result()}
     if e2e is not None:
         line["e2e"] = e2e
@@ -541,7 +548,7 @@ def main():
         for cfg in (5, 3, 2, 1):
             try:
                 r = bench_config(args, cfg, env)
-                line["secondary"].append({k: r[k] for k in ("config", "value", "value_mix_only", "unit", "steps", "ms_per_step",
+                line["secondary"].append({k: r[k] for k in ("config", "run", "value", "value_mix_only", "unit", "steps", "ms_per_step",
                                                              "roofline", "clocks", "gpu_launches", "e2e") if k in r})
             except Exception as ex:       # a secondary record must never take the headline down
                 line["secondary"].append({"config": {"workload": f"config {cfg}"}, "error": repr(ex)})

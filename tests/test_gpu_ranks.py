@@ -131,5 +131,5 @@ def test_bench_rank_launcher_runs_under_torch_distributed_run(cfg, P):
     assert len(lines) == 1
     d = json.loads(lines[0])
     assert d["n_gpus"] == 2 and d["value"] > 0 and d["steps"] == 12 and d["scaling"] == "strong"
-    assert d["config"]["P"] == P and d["config"]["P_per_gpu"] == P // 2
+    assert d["config"]["P"] == P and d["run"]["P_per_gpu"] == P // 2
     assert d["gpu_launches"] > 0 and d["roofline"]["launches"] == 12
