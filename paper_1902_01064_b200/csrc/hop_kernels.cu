@@ -320,29 +320,48 @@ template <bool MOMENTUM, bool DECAY>
 __device__ __forceinline__ void bulk_record_scalar(const BulkRec& r, const int4* __restrict__ ents2, const float* __restrict__ stage,
                                                    int ws, int wd, int nG, float lr, float mu, float lam, float* __restrict__ Xc,
                                                    float* __restrict__ Mc, int64_t P, int lane) {
+    // a lane takes columns cb, cb + 32, cb + 64, cb + 96 per round, so that the table loads and the loop are shared by four
+    // outputs as in the vector form; columns past the tile's width are predicated off (loads included: they could leave the stage)
 #pragma unroll 1
-    for (int c = lane; c < wd; c += 32) {
-        float acc = 0.f;
-        const float* sc = stage + c;
+    for (int cb = lane; cb < wd; cb += 128) {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        const float* sc = stage + cb;
+        const bool on[4] = {true, cb + 32 < wd, cb + 64 < wd, cb + 96 < wd};
         const int4* e = ents2 + (r.ent_begin >> 1);
 #pragma unroll 1
         for (int g = 0; g < r.groups; ++g, e += 2) {
             const int4 e01 = e[0], e23 = e[1];
-            const float v0 = sc[e01.x], v1 = sc[e01.z], v2 = sc[e23.x], v3 = sc[e23.z];
-            acc = fmaf(__int_as_float(e01.y), v0, acc); acc = fmaf(__int_as_float(e01.w), v1, acc);
-            acc = fmaf(__int_as_float(e23.y), v2, acc); acc = fmaf(__int_as_float(e23.w), v3, acc);
-        }
-        if (DECAY && r.self_off >= 0 && r.g_off < 0) acc = fmaf(-lr * lam, sc[r.self_off], acc);
-        if (r.g_off >= 0) {
-            float g = sc[r.g_off];
-            if (DECAY && r.self_off >= 0) g = fmaf(lam, sc[r.self_off], g);
-            if constexpr (MOMENTUM) {
-                g = fmaf(mu, sc[r.g_off + nG * ws], g);
-                Mc[(int64_t)r.worker * P + c] = g;
+            float v[4][4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                v[j][0] = on[j] ? sc[e01.x + 32 * j] : 0.f; v[j][1] = on[j] ? sc[e01.z + 32 * j] : 0.f;
+                v[j][2] = on[j] ? sc[e23.x + 32 * j] : 0.f; v[j][3] = on[j] ? sc[e23.z + 32 * j] : 0.f;
             }
-            acc = fmaf(-lr, g, acc);
+            const float w0 = __int_as_float(e01.y), w1 = __int_as_float(e01.w), w2 = __int_as_float(e23.y), w3 = __int_as_float(e23.w);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                acc[j] = fmaf(w0, v[j][0], acc[j]); acc[j] = fmaf(w1, v[j][1], acc[j]);
+                acc[j] = fmaf(w2, v[j][2], acc[j]); acc[j] = fmaf(w3, v[j][3], acc[j]);
+            }
         }
-        Xc[r.out_off + c] = acc;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (!on[j]) continue;
+            const int c = cb + 32 * j;
+            const float* scj = sc + 32 * j;
+            float a = acc[j];
+            if (DECAY && r.self_off >= 0 && r.g_off < 0) a = fmaf(-lr * lam, scj[r.self_off], a);
+            if (r.g_off >= 0) {
+                float g = scj[r.g_off];
+                if (DECAY && r.self_off >= 0) g = fmaf(lam, scj[r.self_off], g);
+                if constexpr (MOMENTUM) {
+                    g = fmaf(mu, scj[r.g_off + nG * ws], g);
+                    Mc[(int64_t)r.worker * P + c] = g;
+                }
+                a = fmaf(-lr, g, a);
+            }
+            Xc[r.out_off + c] = a;
+        }
     }
 }
 
