@@ -224,7 +224,7 @@ static int set_option_value(hop_ctx* c, int key, double v) {
     return HOP_OK;
 }
 
-static int load_trace_impl(hop_ctx* c, const hop_trace& t, bool rewind);
+static int load_trace_impl(hop_ctx* c, const hop_trace& t, bool rewind, bool validate);
 
 // What plan_level bakes into a loaded level: staged rows, tile width, kernel choice, the gradient rows of the dense path.
 struct PlanShape {
@@ -250,7 +250,7 @@ extern "C" int hop_set_option(hop_ctx* c, int key, double v) {
     if (rc) return rc;
     if (c->loaded && !(plan_shape(c) == before)) {
         // the loaded levels were planned for the old setting: plan and upload them again, keeping the position
-        const int rr = load_trace_impl(c, c->loaded_trace, false);
+        const int rr = load_trace_impl(c, c->loaded_trace, false, false);      // it passed the validation when it was loaded
         if (rr) {            // not plannable under the new setting: keep the old one (tables untouched)
             const std::string why = c->err;
             c->momentum = old_mom; c->weight_decay = old_wd; c->serial = old_serial; c->grad_mode = old_gm; c->mix_kernel = old_mk;
@@ -402,11 +402,11 @@ extern "C" int hop_load_trace(hop_ctx* c, const hop_trace* t) {
     if (!c || !t) return HOP_E_ARG;
     if (!c->bound) HOP_FAIL(c, HOP_E_STATE, "hop_load_trace: bind buffers first");
     if (t->N != c->g.N) HOP_FAIL(c, HOP_E_TRACE, "hop_load_trace: trace has a different number of workers");
-    return load_trace_impl(c, *t, true);
+    return load_trace_impl(c, *t, true, true);
 }
 
 // Validates, plans and uploads; rewind = false keeps the current level (the same trace planned again).
-static int load_trace_impl(hop_ctx* c, const hop_trace& trace, bool rewind) {
+static int load_trace_impl(hop_ctx* c, const hop_trace& trace, bool rewind, bool validate) {
     const hop_trace* t = &trace;
     const int32_t N = t->N, L = t->levels;
     std::vector<int32_t> newest(N, 0);
@@ -417,8 +417,8 @@ static int load_trace_impl(hop_ctx* c, const hop_trace& trace, bool rewind) {
     std::vector<int32_t> taken(c->g.in_idx.size(), -1);
     for (int32_t k = 0; k < L; ++k) {
         const size_t r = (size_t)k * N;
-        const int rc = hop_validate_level(c->g, c->sp, k, &t->op[r], &t->ptr[r], t->nbr.data(), t->ver.data(),
-                                          t->num.data(), &t->den[r], newest, &sent, &taken, c->err);
+        const int rc = !validate ? HOP_OK : hop_validate_level(c->g, c->sp, k, &t->op[r], &t->ptr[r], t->nbr.data(), t->ver.data(),
+                                                                t->num.data(), &t->den[r], newest, &sent, &taken, c->err);
         if (rc) return rc;
         hop_build_level(c->g, c->s, k, &t->op[r], &t->ptr[r], t->nbr.data(), t->ver.data(), t->num.data(), &t->den[r], levels[k]);
         const int rc2 = plan_level(c, levels[k]);

@@ -651,12 +651,13 @@ def test_options_set_after_load_trace_plan_the_levels_again():
 
 
 def test_option_change_in_the_middle_of_a_run_keeps_the_position():
-    w = workload(3, P=1024, iters=20)
+    w = workload(3, op.REUSE, P=1024, iters=20)
     x0 = np.stack([w.p0() + w.perturbation(i) for i in range(w.N)])
     ref = GpuRun(w, x0=x0).run(w.iters)
     g = GpuRun(w, x0=x0)
     g.run(9)
-    g.h.set_option(hop.OPT_MIX_KERNEL, hop.MIX_STAGED)        # planned again at level 9
+    g.h.set_option(hop.OPT_STALE_REDUCE, hop.STALE_NEW_ONLY)  # a protocol option: acts on traces simulated or loaded later,
+    g.h.set_option(hop.OPT_MIX_KERNEL, hop.MIX_STAGED)        # not on the loaded one, which is planned again at level 9
     assert g.h.level_stats(12)["kernel"] == hop.MIX_STAGED
     got = g.run(w.iters - 9)
     for i in range(w.N):
