@@ -488,6 +488,8 @@ def bench_config(args, cfg, env):
             "run": {"P_per_gpu": w.P, "parallelism": f"column-sharded x{world}", "trace_passes": steps / w.iters,
                     "timed_levels": f"{timed_levels[0]}..{timed_levels[-1]}" if steps <= w.iters else f"whole trace x{steps / w.iters:.2f}",
                     "protocol_sim_ms": sim_ms,
+                    "records_timed": {"normal": normal_timed, "jump": int(sum(int((tr["op"][k] == 2).sum()) for k in timed_levels)),
+                                      "idle": int(sum(int((tr["op"][k] == 0).sum()) for k in timed_levels))},
                     "launch": "hop_run: CUDA graph replay of the trace" if use_graph else "hop_step per level"},
             "roofline": roofline, "gpu_launches": int(launches), "clocks": sampler.result()}
     if e2e is not None:
