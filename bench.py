@@ -210,6 +210,7 @@ def run_reference(args):
         return
     from paper_1902_01064_b200 import inputs
     w = inputs.make_workload(args.config)
+    w.stale_reduce = 1 if args.stale_reduce == "reuse" else 0
     vals = []
     steps, warm = max(1, min(args.steps, 3)), min(args.warmup, 1)
     for it in range(warm + steps):
@@ -261,6 +262,7 @@ def bench_config(args, cfg, env):
     world, rank, local, dist = env["world"], env["rank"], env["local"], env["dist"]
     steps = args.steps
     w = inputs.make_workload(cfg, P=args.P)
+    w.stale_reduce = 1 if args.stale_reduce == "reuse" else 0
     P_global = w.P
     lo, hi = shard_columns(P_global, world, rank)
     p0 = w.p0()[lo:hi].copy()
@@ -507,6 +509,8 @@ def main():
     ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"], help="process-group backend when WORLD_SIZE > 1")
     ap.add_argument("--P", type=int, default=None, help="override the parameter count (profiling on a small case)")
     ap.add_argument("--mix-kernel", type=int, default=0)
+    ap.add_argument("--stale-reduce", default="new_only", choices=["new_only", "reuse"],
+                    help="which updates inside the staleness bound enter a Reduce (default: Eq. 2 as printed)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-secondary", action="store_true")
@@ -556,6 +560,7 @@ def main():
                 line["secondary"].append({"config": {"workload": f"config {cfg}"}, "error": repr(ex)})
     if rank == 0 and not args.no_cpu_baseline and world == 1:
         wf = inputs.make_workload(headline_cfg, P=args.P)
+        wf.stale_reduce = 1 if args.stale_reduce == "reuse" else 0
         v, desc = oracle_sample(wf)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
         try:
