@@ -395,7 +395,7 @@ mix_bulk_kernel(float* __restrict__ X, float* __restrict__ M, const float* __res
     const int ws = ALIGNED ? w : w + 4;                    // floats per staged row
     const int64_t stage_floats = (int64_t)rows * ws;
     const int64_t tiles = (P + w - 1) / w;
-    launch_dependents();     // a kernel behind that was launched as a dependent (the sparse apply) may fetch its static data
+    launch_dependents();     // a kernel behind that was launched as a dependent (a CSR margin kernel) may fetch its static data
     if (!(ALIGNED && early_x)) dependency_wait();
     if (tid == 0) {
         for (int s = 0; s < kBulkStages; ++s) { mbar_init(&full[s], kProducerWarps); mbar_init(&empty[s], kConsumerWarps); }
