@@ -783,3 +783,40 @@ def test_bulk_kernel_with_unaligned_rows_equals_the_general_kernel_bitwise(P):
         assert torch.equal(a.M, b.M)
         a.h.close()
         b.h.close()
+
+
+def test_a_level_with_more_distinct_slices_than_shared_memory_can_stage_is_refused():
+    # 128 workers on a complete graph, 64 versions each in the ring: at level 63 every worker takes a different version
+    # from every neighbour, 8192 distinct slices in one level.  No tile width fits: hop_load_trace says so (and nothing
+    # is launched); a smaller trace then loads into the same context.
+    N, s, P, L = 128, 63, 16, 64
+    ptr, idx = inputs.graph_to_csr(inputs.complete(N))
+    h = hop.Hop(ptr, idx, N, P, s, N - 1, 0)                       # one usable in-neighbour (the own update) suffices
+    h.set_option(hop.OPT_WEIGHT_MODE, hop.W_STALE_LINEAR)
+    h.set_option(hop.OPT_GRAD_MODE, hop.GRAD_SYNTHETIC)
+    X = torch.zeros((N, s + 1, P), dtype=torch.float32, device=DEV)
+    G = torch.zeros((N, P), dtype=torch.float32, device=DEV)
+    h.bind_buffers(X, None, G, torch.cuda.current_stream().cuda_stream)
+    ops = np.full((L, N), op.NORMAL, np.int32)
+    t_ptr, nbr, ver, num = [0], [], [], []
+    den = np.zeros((L, N), np.int32)
+    for k in range(L):
+        for i in range(N):
+            rec = [(i, k)] if k < L - 1 else [(j, k if j == i else k - ((i + j) % 64)) for j in range(N)]
+            for (j, v) in rec:
+                nbr.append(j); ver.append(v); num.append(v - (k - s) + 1)
+            den[k, i] = sum(num[t_ptr[-1]:])
+            t_ptr.append(len(nbr))
+    big = hop.Trace.from_arrays(ops, np.asarray(t_ptr, np.int64), nbr, ver, num, den)
+    with pytest.raises(hop.HopError) as e:
+        h.load_trace(big)
+    assert e.value.code == hop.E_UNSUPPORTED and "distinct slices" in str(e.value)
+    with pytest.raises(hop.HopError) as e:
+        h.step()                                                   # nothing is loaded
+    assert e.value.code == hop.E_STATE
+    small = hop.Trace.from_arrays(ops[:3], np.asarray(t_ptr[:3 * N + 1], np.int64), nbr[:3 * N], ver[:3 * N], num[:3 * N], den[:3])
+    h.load_trace(small)
+    for _ in range(3):
+        h.step()
+    assert h.read_status() == 0
+    h.close()
