@@ -820,3 +820,14 @@ def test_a_level_with_more_distinct_slices_than_shared_memory_can_stage_is_refus
         h.step()
     assert h.read_status() == 0
     h.close()
+
+
+def test_reduce_set_study_runs_and_trains():
+    from paper_1902_01064_b200 import study
+    rows = study.reduce_set_study(P=2048, iters=200)
+    assert len(rows) == 4
+    start = 1.0                                        # hinge loss at p_0 = 0
+    for reduce_name, weights, loss, spread, entries in rows:
+        assert np.isfinite(loss) and loss < start and spread < 1.0
+    by = {(r[0], r[1]): r for r in rows}
+    assert by[("since previous Recv", "Eq. 2")][4] < by[("all inside the bound", "Eq. 2")][4]     # fewer terms per Reduce
