@@ -831,3 +831,44 @@ def test_reduce_set_study_runs_and_trains():
         assert np.isfinite(loss) and loss < start and spread < 1.0
     by = {(r[0], r[1]): r for r in rows}
     assert by[("since previous Recv", "Eq. 2")][4] < by[("all inside the bound", "Eq. 2")][4]     # fewer terms per Reduce
+
+
+@pytest.mark.parametrize("cfg,P,kernel", [(3, 5000, hop.MIX_BULK), (3, 4999, hop.MIX_BULK), (3, 4999, hop.MIX_STAGED),
+                                          (4, 3001, hop.MIX_BULK), (5, 1536, hop.MIX_TENSOR), (2, 4098, hop.MIX_AUTO)])
+def test_no_kernel_writes_outside_the_bound_buffers(cfg, P, kernel):
+    # X, M and G are carved out of larger allocations whose margins hold a sentinel; after a full run (unaligned row
+    # lengths, ragged last tiles, momentum, jumps, the tensor path, the sparse apply) every margin is untouched.
+    w = workload(cfg, P=P, iters=12)
+    S, guard, sentinel = w.s + 1, 4096, -12345.5
+    def carve(n):
+        if n == 0:
+            return None, None
+        whole = torch.full((guard + n + guard,), sentinel, dtype=torch.float32, device=DEV)
+        return whole, whole[guard:guard + n]
+    wx, X = carve(w.N * S * P)
+    wm, M = carve(w.N * P if w.momentum else 0)
+    wg, G = carve(0 if w.grad_mode == inputs.GRAD_SVM_CSR else w.N * P)
+    X.zero_()
+    if M is not None:
+        M.zero_()
+    if G is not None:
+        G.zero_()
+    h = hop.from_workload(w, kernel)
+    h.bind_buffers(X, M, G, torch.cuda.current_stream().cuda_stream)
+    keep = []
+    if w.grad_mode == inputs.GRAD_SVM_CSR:
+        keep = [torch.from_numpy(a).to(DEV) for a in (w.svm.row_ptr, w.svm.col, w.svm.val, w.svm.y)]
+        h.bind_svm_csr(*keep, w.svm.rows_per_worker, w.svm.batch)
+    h.load_trace(h.sim_run(w.ticks, w.iters))
+    if kernel != hop.MIX_AUTO:
+        assert h.level_stats(2)["kernel"] == kernel
+    h.write_params(-1, 0, w.p0())
+    for _ in range(w.iters):
+        h.step()
+    assert h.read_status() == 0
+    torch.cuda.synchronize()
+    for whole in (wx, wm, wg):
+        if whole is not None:
+            assert bool((whole[:guard] == sentinel).all()) and bool((whole[-guard:] == sentinel).all())
+    assert bool(torch.isfinite(X).all())
+    h.close()
