@@ -872,3 +872,24 @@ def test_no_kernel_writes_outside_the_bound_buffers(cfg, P, kernel):
             assert bool((whole[:guard] == sentinel).all()) and bool((whole[-guard:] == sentinel).all())
     assert bool(torch.isfinite(X).all())
     h.close()
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3])
+def test_full_size_graph_replay_equals_step_by_step(cfg):
+    # bench.py times configurations 1-3 through hop_run (one replayed CUDA graph per pass of the trace, with the
+    # dependent launches inside it); at full size that path must give what the step-by-step path gives, which the
+    # full-size tests above compare with the oracle
+    w = inputs.make_workload(cfg)
+    ref = GpuRun(w).run(w.iters)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        g = GpuRun(w)
+        g.h.run(w.iters)
+        got = [g.h.read_params(i) for i in range(w.N)]
+        assert g.h.read_status() == 0
+        g.h.close()
+    for i in range(w.N):
+        if cfg == 2:                                   # float atomics in the sparse apply: order may differ
+            assert np.abs(got[i] - ref[i]).max() <= 1e-5 * (np.abs(ref[i]).max() + 1e-30)
+        else:
+            assert np.array_equal(got[i], ref[i])
