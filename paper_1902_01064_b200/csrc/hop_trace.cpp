@@ -86,11 +86,14 @@ int hop_validate_level(const HopGraph& g, const HopSimParams& p, int32_t level, 
         if (e - a > d) return fail(i, "more consumed updates than in-neighbours");
         int64_t sum = 0;
         bool own = false;
+        const auto nb_begin = g.in_idx.begin() + g.in_ptr[i], nb_end = g.in_idx.begin() + g.in_ptr[i + 1];
+        auto walk = nb_begin;            // records usually list neighbours in ascending order, like the graph: one merge pass
         for (int64_t t = a; t < e; ++t) {
             const int32_t j = nbr[t], v = ver[t];
             if (j < 0 || j >= N) return fail(i, "neighbour id out of range");
-            const auto edge = std::lower_bound(g.in_idx.begin() + g.in_ptr[i], g.in_idx.begin() + g.in_ptr[i + 1], j);
-            if (edge == g.in_idx.begin() + g.in_ptr[i + 1] || *edge != j)
+            while (walk != nb_end && *walk < j) ++walk;
+            const auto edge = (walk != nb_end && *walk == j) ? walk : std::lower_bound(nb_begin, nb_end, j);
+            if (edge == nb_end || *edge != j)
                 return fail(i, "consumed worker " + std::to_string(j) + " is not an in-neighbour");
             if (seen[j] == i) return fail(i, "neighbour consumed twice");
             seen[j] = i;
@@ -127,6 +130,9 @@ void hop_build_level(const HopGraph& g, int32_t s, int32_t level, const int32_t*
     const int32_t N = g.N, S = s + 1;
     std::vector<int32_t> slice_of((size_t)N * S, -1);
     out = HopLevelHost();
+    const size_t n_ent = (size_t)(ptr[N] - ptr[0]) + 3 * (size_t)N;      // entries plus per-record padding
+    out.ents.reserve(n_ent); out.ent_slice.reserve(n_ent); out.ent_num.reserve(n_ent);
+    out.recs.reserve(N); out.rec_den.reserve(N); out.grad_workers.reserve(N); out.src_row.reserve(std::min(n_ent, (size_t)N * S));
     for (int32_t i = 0; i < N; ++i) {
         if (op[i] == HOP_OP_IDLE) continue;
         HopRecord r{};
