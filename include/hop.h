@@ -137,6 +137,7 @@ typedef enum hop_option {
     HOP_OPT_LOSS = 14,        /* hop_loss of the SVM modes (default HINGE; the paper's runs used LOG, Section 7.2)    */
     HOP_OPT_APPROACH = 15,    /* hop_approach (default PARALLEL, the paper's choice, Section 3.2)                     */
     HOP_OPT_STALE_REDUCE = 16,/* hop_stale_reduce (default NEW_ONLY: Eq. 2 / Fig. alg3 as printed)                    */
+    HOP_OPT_NVTX = 17,        /* 1: an NVTX range "hop level k" on the host timeline around each level's launches     */
     HOP_OPT_BACKUP_OF_WORKER = 1000 /* key = 1000 + i sets N_buw(i) of one worker (Fig. alg4)       */
 } hop_option;
 

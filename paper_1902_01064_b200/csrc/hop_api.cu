@@ -1,8 +1,10 @@
 // C ABI of libhop_b200.so: context, options, buffer binding, trace upload, level execution.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <algorithm>
 #include <cmath>
+#include <cstdio>
 #include <cstring>
 #include <string>
 #include <map>
@@ -46,6 +48,7 @@ struct hop_ctx {
     int32_t tc_slots = 0;
     bool tc_maps_ready = false;
     // hop_run: instantiated CUDA graphs of level ranges, keyed by (first level, count)
+    bool nvtx = false;              // one NVTX range per level around the enqueue calls (tracing aid)
     bool use_graph = true;
     struct Graph { cudaGraphExec_t exec; int64_t launches; };
     std::map<std::pair<int32_t, int32_t>, Graph> graphs;
@@ -162,6 +165,7 @@ extern "C" int hop_destroy(hop_ctx* c) {
 
 static int set_option_value(hop_ctx* c, int key, double v) {
     if (key == HOP_OPT_USE_GRAPH) { c->use_graph = v != 0.0; return HOP_OK; }
+    if (key == HOP_OPT_NVTX) { c->nvtx = v != 0.0; return HOP_OK; }
     if (key == HOP_OPT_NOTIFY_ACK) { c->sp.notify_ack = v != 0.0; return HOP_OK; }
     if (key == HOP_OPT_WEIGHT_DECAY) {
         if (v < 0) HOP_FAIL(c, HOP_E_ARG, "hop_set_option: weight decay must be non-negative");
@@ -512,7 +516,19 @@ static int ensure_tc_maps(hop_ctx* c) {
 // phase 2: the rest (SVM modes start from the margins the caller has summed over the column shards).
 // chained: the operation in front of this level on the stream is the previous level of the same hop_run call (a kernel of
 // this library), not something the caller enqueued.
+struct NvtxLevelRange {         // "hop level k" on the host timeline while the level's kernels are enqueued
+    bool on;
+    NvtxLevelRange(bool enabled, int level, int phase) : on(enabled) {
+        if (!on) return;
+        char name[48];
+        snprintf(name, sizeof name, phase == 0 ? "hop level %d" : (phase == 1 ? "hop level %d (begin)" : "hop level %d (end)"), level);
+        nvtxRangePushA(name);
+    }
+    ~NvtxLevelRange() { if (on) nvtxRangePop(); }
+};
+
 static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, const TcPtrs& tc, int phase = 0, bool chained = false) {
+    NvtxLevelRange range(c->nvtx, lv.level, phase);
     size_t t0 = 0, t1 = 0;
     HopLaunchCfg cfg{};
     cfg.X = c->X; cfg.M = c->M; cfg.G = c->G; cfg.P = c->P; cfg.N = c->g.N; cfg.s = c->s;

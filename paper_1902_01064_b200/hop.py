@@ -22,7 +22,7 @@ GRAD_EXTERNAL, GRAD_SYNTHETIC, GRAD_SVM_DENSE, GRAD_SVM_CSR = 0, 1, 2, 3
 MIX_AUTO, MIX_STAGED, MIX_BULK, MIX_TENSOR = 0, 1, 2, 3
 (OPT_MAX_IG, OPT_LR, OPT_MOMENTUM, OPT_WEIGHT_MODE, OPT_GRAD_MODE, OPT_GRAD_SEED, OPT_GRAD_SIGMA,
  OPT_MIX_KERNEL, OPT_COL_OFFSET, OPT_USE_GRAPH, OPT_BACKUP_MODE, OPT_NOTIFY_ACK, OPT_WEIGHT_DECAY, OPT_LOSS,
- OPT_APPROACH, OPT_STALE_REDUCE) = range(1, 17)
+ OPT_APPROACH, OPT_STALE_REDUCE, OPT_NVTX) = range(1, 18)
 STALE_NEW_ONLY, STALE_REUSE = 0, 1
 LOSS_HINGE, LOSS_LOG = 0, 1
 APPROACH_PARALLEL, APPROACH_SERIAL = 0, 1
