@@ -217,7 +217,12 @@ int hop_newest_version(hop_ctx* ctx, int32_t worker, int32_t* version);
 int hop_set_level(hop_ctx* ctx, int32_t level);
 /* Executes the next level k of the loaded trace for all N workers: gradient kernels on slot k,
  * then the fused gather-mix-update writing slot k+1, then (CSR SVM) the sparse apply.
- * Asynchronous; HOP_E_STATE past the end of the trace. */
+ * Asynchronous; HOP_E_STATE past the end of the trace.
+ * Ordering on the stream: the first kernel of a call waits for everything enqueued before the call; the kernels
+ * of the call are ordered among themselves, except that the mix-update kernel may read X and M (which the
+ * library's gradient kernels do not write) while the level's gradient kernel is still finishing -- it waits for
+ * that kernel before it reads G and before it writes anything.  With HOP_GRAD_EXTERNAL every kernel is fully
+ * ordered behind the caller's work. */
 int hop_step(hop_ctx* ctx);
 /* Split-phase form of hop_step for a parameter vector sharded by columns over several contexts (one per GPU):
  * mixing and the dense / synthetic gradients are separable by column, but an SVM margin a_r . x needs all columns.
@@ -232,7 +237,9 @@ int hop_step_end(hop_ctx* ctx);
  * stream, the levels are captured once into a CUDA graph (cached per (first level, n_levels); dropped
  * by any bind / option / trace change) and replayed, which removes most of the per-kernel launch cost
  * that dominates small problems.  Falls back to a plain loop of hop_step on the default stream, while
- * timing is enabled, with HOP_GRAD_EXTERNAL, or with HOP_OPT_USE_GRAPH = 0.  Asynchronous. */
+ * timing is enabled, with HOP_GRAD_EXTERNAL, or with HOP_OPT_USE_GRAPH = 0.  Asynchronous.
+ * Inside one call the CSR margin kernel of every level but the first may fetch its row data (row_ptr, col, val:
+ * read-only to the library) while the previous level's last kernel is finishing. */
 int hop_run(hop_ctx* ctx, int32_t n_levels);
 /* Same for one level handed in from the host (streaming use: the protocol decides level by
  * level): validates the records, uploads them from a pinned staging buffer, executes the level,
