@@ -87,3 +87,20 @@ def test_trace_roundtrip():
     for k in ("op", "ptr", "nbr", "ver", "num", "den"):
         assert np.array_equal(a[k], b[k])
     assert t2.dims()[:3] == (30, 32, len(a["nbr"]))
+
+
+def test_python_constants_match_the_header():
+    """hop.py repeats the header's enumerators by hand: they must not drift apart."""
+    text = open(os.path.join(ROOT, "include", "hop.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    enums = {name: int(val) for name, val in re.findall(r"\b(HOP_[A-Z0-9_]+)\s*=\s*(-?\d+)", text)}
+    assert len(enums) > 45
+    missing = []
+    for name, val in enums.items():
+        py = name[len("HOP_"):]
+        if not hasattr(hop, py):
+            missing.append(name)
+            continue
+        assert getattr(hop, py) == val, name
+    assert not missing, missing
+    assert hop.STATIC_MAX_ROWS == int(re.search(r"#define HOP_STATIC_MAX_ROWS (\d+)", text).group(1))
