@@ -535,3 +535,33 @@ def test_notify_ack_chain_reaches_both_bounds_of_table1_exactly():
                 top[i] = max(top[i], p.Iter[i])
     op.simulate(n_in, ticks, 8, notify_ack=True, on_round=chk)
     assert top == [3, 1, 0]
+
+
+@pytest.mark.parametrize("case,s,b,max_ig", [("a", 4, 0, 4), ("b", 4, 1, 5)])
+def test_skipping_prose_examples_lead_then_as_much_again_after_the_jump(case, s, b, max_ig):
+    """Section 5, the two examples of the skipping figure: three workers, A (worker 0) always slow.  Without skipping B and C
+    get `lead` iterations ahead and wait; when A jumps to their iteration they run on for as many iterations again
+    before A's next progress.  (a) the lead comes from the token queues of a staleness run (max_ig = s = 4);
+    (b) from max_ig = 5 with one backup worker."""
+    g = golden()
+    lead, more = int(g[f"skip_example.{case}.lead"]), int(g[f"skip_example.{case}.more_after_jump"])
+    if case == "b":
+        assert max_ig == int(g["skip_example.b.max_ig"])
+    slow = 1000
+    ticks = np.ones((3, 40), np.uint64)
+    ticks[0, :] = slow
+    tops = {}
+
+    def chk(p):
+        w = int(p.now // slow)                      # which of A's computes is running
+        tops[w] = max(tops.get(w, 0), p.Iter[1], p.Iter[2])
+    no_skip = {}
+    op.simulate(inputs.complete(3), ticks[:, :12], 12, s=s, b=b, max_ig=max_ig, max_skip=0, weight_mode=op.STALE_LINEAR,
+                on_round=lambda p: no_skip.__setitem__(int(p.now // slow), max(no_skip.get(int(p.now // slow), 0), p.Iter[1])))
+    assert no_skip[0] == lead and no_skip[1] == lead + 1      # dragged along: one more iteration per step of A
+    tr = op.simulate(inputs.complete(3), ticks, 40, s=s, b=b, max_ig=max_ig, max_skip=s + 1, weight_mode=op.STALE_LINEAR, on_round=chk)
+    assert tops[0] == lead                                      # before A's first step: the bounded lead
+    assert tops[1] == lead + more                               # A jumped to their iteration: as many iterations again
+    assert tops[2] == lead + 2 * more
+    jumps = [(k, i) for k in range(40) for i in range(3) if tr.op[k, i] == op.JUMP]
+    assert jumps and all(i == 0 for _, i in jumps)
