@@ -573,6 +573,10 @@ def main():
                                                  "sample": f"same update rules on {allc[2]} columns dealt to {allc[1]} processes "
                                                            f"({allc[3]:.2f} s), protocol simulation serial"}
     if rank == 0:
+        # the paper reports no number for this path; its own speedups, with their hardware, as context only
+        line["paper_context"] = ("Hop paper, Section 7: CPU cluster, 16 workers on 4 machines, 1 Gbit/s Ethernet, TensorFlow -- one backup "
+                                 "worker: up to 1.81x iteration speed under a random 6x slowdown; skipping iterations: a 4x straggler's "
+                                 "effect on the iteration time cut from 3.9x to 1.1x.  Not comparable with worker-iterations/s on one GPU.")
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
