@@ -253,10 +253,15 @@ int hop_step_host(hop_ctx* ctx, const int32_t* op, const int64_t* ptr, const int
  * stage, on the tensor pipeline) is bounded; a kernel that gives up records the first such event and returns, so
  * the context and the GPU stay usable.  0 = nothing happened (HOP_OK); otherwise HOP_E_DEVICE, the word has a code
  * in its top byte (1: mix_bulk_kernel, a tile's copies did not arrive; 2: mix_bulk_kernel, no stage became free;
- * 3: mix_dense_tc_kernel, a pipeline wait ran out) and a detail in the low 24 bits (tile index or wait site), and
+ * 3: mix_dense_tc_kernel, a pipeline wait ran out; 4: only in the bounds-checked build of the library, an access
+ * outside the bound buffers was refused) and a detail in the low 24 bits (tile index or site), and
  * hop_last_error names it.  The parameters written by that level are then undefined.  The word is sticky until
  * hop_clear_status. */
 int hop_read_status(hop_ctx* ctx, int32_t* device_error_word);
+/* 1 if this library is the bounds-checked build (compiled with -DHOP_CHECKED: global-memory sources of the mix kernels'
+ * copies and the gathers / atomics of the CSR SVM kernels are tested against the bound buffers X, M, G; an access outside
+ * them is refused and recorded as status code 4; hop_run does not replay graphs), else 0.  Touches no GPU. */
+int hop_build_is_checked(void);
 /* Resets the device-side error word (asynchronous on the bound stream). */
 int hop_clear_status(hop_ctx* ctx);
 /* Self-test of that mechanism: launches one warp that waits on a barrier nothing completes, gives up after `polls`

@@ -536,7 +536,8 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, c
     cfg.use_g = c->grad_mode != HOP_GRAD_SVM_CSR;
     cfg.sm_count = c->sm_count; cfg.err_word = c->d_err; cfg.stream = c->stream;
     cfg.table_smem = L.table_smem; cfg.n_ents = (int32_t)L.ents.size();
-    int e = 0;
+    int e = hop_checked_set_fence(cfg);
+    if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("checked build, buffer ranges: ") + cudaGetErrorString((cudaError_t)e));
     bool grad_kernel_in_front = false;      // a gradient kernel of this library was launched by this call, right before the mix
     if (L.nG > 0 && c->grad_mode != HOP_GRAD_EXTERNAL) {
         HOP_SPAN_BEGIN();
@@ -668,7 +669,8 @@ extern "C" int hop_run(hop_ctx* c, int32_t n_levels) {
     const int32_t first = c->level;
     // Graph replay needs a capturable stream (not the legacy default stream), no per-kernel event timing,
     // and a gradient source that is part of the library (an external G changes between levels).
-    const bool graph = c->use_graph && c->stream != nullptr && !c->timing && c->grad_mode != HOP_GRAD_EXTERNAL && n_levels > 1;
+    const bool graph = c->use_graph && c->stream != nullptr && !c->timing && c->grad_mode != HOP_GRAD_EXTERNAL && n_levels > 1 &&
+                       !hop_checked_build();      // the checked build copies its buffer ranges from pageable memory: not capturable
     if (!graph) {
         for (int32_t k = first; k < first + n_levels; ++k)
             if ((rc = enqueue_level(c, k, k > first))) return rc;
@@ -828,13 +830,16 @@ extern "C" int hop_read_status(hop_ctx* c, int32_t* word) {
     HOP_CUDA(c, cudaMemcpy(word, c->d_err, sizeof(int32_t), cudaMemcpyDeviceToHost));
     if (*word != 0) {
         static const char* what[] = {"unknown", "mix_bulk_kernel: a tile's copies did not arrive", "mix_bulk_kernel: no stage became free",
-                                     "mix_dense_tc_kernel: a pipeline wait ran out"};
+                                     "mix_dense_tc_kernel: a pipeline wait ran out",
+                                     "checked build: an access outside the bound buffers was refused"};
         const int code = (*word >> 24) & 0xff;
-        HOP_FAIL(c, HOP_E_DEVICE, std::string("a kernel gave up waiting -- ") + what[code >= 1 && code <= 3 ? code : 0] +
+        HOP_FAIL(c, HOP_E_DEVICE, std::string("a kernel reported -- ") + what[code >= 1 && code <= 4 ? code : 0] +
                                   " (status word " + std::to_string(*word) + ", detail " + std::to_string(*word & 0xffffff) + ")");
     }
     return HOP_OK;
 }
+
+extern "C" int hop_build_is_checked(void) { return hop_checked_build() ? 1 : 0; }
 
 extern "C" int hop_clear_status(hop_ctx* c) {
     if (!c) return HOP_E_ARG;

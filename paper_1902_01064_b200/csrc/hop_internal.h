@@ -146,6 +146,8 @@ int hop_launch_svm_csr_apply(const HopLaunchCfg& c, const HopLevelDev& lv, const
 // serial approach, dense gradients: x_k <- x_k - lr * d in place for the level's NORMAL workers
 int hop_launch_apply_dense(const HopLaunchCfg& c, const HopLevelDev& lv);
 bool hop_svm_dense_is_fused(int64_t P, int32_t B);   // the dense SVM gradient of a level is one launch instead of two
+int hop_checked_set_fence(const HopLaunchCfg& c);     // checked build only (no-op otherwise): bound-buffer ranges for the kernels
+bool hop_checked_build();
 int hop_launch_wait_selftest(int32_t* err_word, uint32_t polls, int32_t detail, void* stream);
 int hop_mix_smem_budget(int kernel);   // usable dynamic shared memory per CTA for the kernel
 int hop_mix_stages(int kernel);

@@ -28,7 +28,30 @@ constexpr int kBulkThreads = 32 * (kConsumerWarps + kProducerWarps);
 constexpr int kBulkStages = 2;
 constexpr uint32_t kSpinLimit = 1u << 22;
 
-enum : int32_t { ERR_FULL_WAIT = 1 << 24, ERR_EMPTY_WAIT = 2 << 24 };
+enum : int32_t { ERR_FULL_WAIT = 1 << 24, ERR_EMPTY_WAIT = 2 << 24, ERR_BOUNDS = 4 << 24 };
+
+// Checked build (-DHOP_CHECKED, a separate library used by the tests; compute-sanitizer's place): every global-memory
+// source of a bulk copy or cp.async, and every gather of the SVM kernels, is first tested against the bound buffers
+// X, M and G.  An access outside them is recorded (status code 4, detail = which site) and skipped, never made.
+#ifdef HOP_CHECKED
+struct HopFence { const char* lo[3]; const char* hi[3]; int32_t* err; };
+__device__ HopFence g_fence;
+__device__ __forceinline__ bool fence_ok(const void* p, size_t bytes, int site) {
+    const char* a = static_cast<const char*>(p);
+#pragma unroll
+    for (int k = 0; k < 3; ++k)
+        if (g_fence.lo[k] != nullptr && a >= g_fence.lo[k] && a + bytes <= g_fence.hi[k]) return true;
+    if (g_fence.err != nullptr) atomicCAS(g_fence.err, 0, ERR_BOUNDS | site);
+    return false;
+}
+#define HOP_FENCE(ptr, bytes, site) do { if (!fence_ok((ptr), (bytes), (site))) return; } while (0)
+#define HOP_FENCE_OR(ptr, bytes, site, fallback) (fence_ok((ptr), (bytes), (site)) ? *(ptr) : (fallback))
+#define HOP_FENCED(ptr, bytes, site) fence_ok((ptr), (bytes), (site))
+#else
+#define HOP_FENCE(ptr, bytes, site) do { } while (0)
+#define HOP_FENCE_OR(ptr, bytes, site, fallback) (*(ptr))
+#define HOP_FENCED(ptr, bytes, site) true
+#endif
 
 // ------------------------------------------------------------------------------------------------
 // Consumer math shared by both mix kernels: one warp produces the tile of one record.
@@ -131,9 +154,11 @@ __device__ __forceinline__ void reduce_apply_record(const HopRecord& r, const Ho
 // a multiple of 4: 4-byte copies (the rows are not 16-byte aligned in global memory, the staged copy is), vector
 // math, scalar stores.  MODE 2: scalar everything (tile widths below 32 that are not multiples of 4).
 __device__ __forceinline__ void cp_async_4(float* dst, const float* src) {
+    HOP_FENCE(src, 4, 1);
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_16(float* dst, const float* src) {
+    HOP_FENCE(src, 16, 2);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
 }
 template <int MODE, bool MOMENTUM, bool DECAY>
@@ -220,6 +245,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     return false;
 }
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    HOP_FENCE(src, bytes, 3);      // a skipped copy leaves the barrier short: the bounded waits end the kernel
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
@@ -664,11 +690,11 @@ svm_margin_csr_kernel(const float* __restrict__ X, int64_t P, int S, HopLevelDev
     double m = 0.0;
     float xv[kCsrPrefetch];
 #pragma unroll
-    for (int q = 0; q < kCsrPrefetch; ++q) xv[q] = (t0 + 32 * q < t1) ? x[pc[q]] : 0.f;     // the gathers in flight together
+    for (int q = 0; q < kCsrPrefetch; ++q) xv[q] = (t0 + 32 * q < t1) ? HOP_FENCE_OR(x + pc[q], 4, 4, 0.f) : 0.f;   // the gathers in flight together
 #pragma unroll
     for (int q = 0; q < kCsrPrefetch; ++q)
         if (t0 + 32 * q < t1) m += (double)pv[q] * (double)xv[q];                           // a lane's elements in their order
-    for (int64_t t = t0 + 32 * kCsrPrefetch; t < t1; t += 32) m += (double)val[t] * (double)x[col[t]];
+    for (int64_t t = t0 + 32 * kCsrPrefetch; t < t1; t += 32) m += (double)val[t] * (double)HOP_FENCE_OR(x + col[t], 4, 4, 0.f);
     m = warp_sum(m);
     if (lane == 0) {
         if (margins_out) margins_out[(int64_t)worker * B + r] = m;     // partial margin over this shard's columns
@@ -813,8 +839,9 @@ svm_csr_apply_kernel(float* __restrict__ X, int64_t P, int S, float lr, HopLevel
     const float scale = -lr * cf;
 #pragma unroll
     for (int q = 0; q < kCsrPrefetch; ++q)
-        if (pc[q] >= 0) atomicAdd(x + pc[q], scale * pv[q]);
-    for (int64_t t = t0 + 32 * kCsrPrefetch; t < t1; t += 32) atomicAdd(x + col[t], scale * val[t]);
+        if (pc[q] >= 0 && HOP_FENCED(x + pc[q], 4, 5)) atomicAdd(x + pc[q], scale * pv[q]);
+    for (int64_t t = t0 + 32 * kCsrPrefetch; t < t1; t += 32)
+        if (HOP_FENCED(x + col[t], 4, 5)) atomicAdd(x + col[t], scale * val[t]);
 }
 
 // Serial approach (Compute, Apply, then Send): x_k <- x_k - lr * d in place for the level's NORMAL workers, with
@@ -857,6 +884,29 @@ size_t staged_smem(const HopLaunchCfg& c, const HopLevelDev& lv) {
 }
 
 }  // namespace
+
+// Checked build: tells the kernels which address ranges are the bound buffers (stream-ordered, before the level's launches).
+int hop_checked_set_fence(const HopLaunchCfg& c) {
+#ifdef HOP_CHECKED
+    HopFence f{};
+    const size_t ring = (size_t)c.N * (c.s + 1) * c.P * sizeof(float), per = (size_t)c.N * c.P * sizeof(float);
+    f.lo[0] = reinterpret_cast<const char*>(c.X); f.hi[0] = f.lo[0] + ring;
+    f.lo[1] = reinterpret_cast<const char*>(c.M); f.hi[1] = c.M ? f.lo[1] + per : nullptr;
+    f.lo[2] = reinterpret_cast<const char*>(c.G); f.hi[2] = c.G ? f.lo[2] + per : nullptr;
+    f.err = c.err_word;
+    return (int)cudaMemcpyToSymbolAsync(g_fence, &f, sizeof f, 0, cudaMemcpyHostToDevice, (cudaStream_t)c.stream);
+#else
+    (void)c;
+    return 0;
+#endif
+}
+bool hop_checked_build() {
+#ifdef HOP_CHECKED
+    return true;
+#else
+    return false;
+#endif
+}
 
 // One launch for margins + coefficients + gradient when a worker's minibatch is small (B * P floats, read twice).
 bool hop_svm_dense_is_fused(int64_t P, int32_t B) { return B <= 4096 && (int64_t)B * P <= 65536; }

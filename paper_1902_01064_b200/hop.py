@@ -9,7 +9,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libhop_b200.so")
+# HOP_B200_LIBRARY selects another build of the same sources (the bounds-checked one the tests use)
+LIB_PATH = os.environ.get("HOP_B200_LIBRARY") or os.path.join(_HERE, "libhop_b200.so")
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_1902_01064_b200.build` "
                       "(the Hop hot path has no CPU fallback)")
@@ -57,6 +58,7 @@ SIGNATURES = {
     "hop_step_host": [_p, _p, _p, _p, _p, _p, _p, _p, _i64],
     "hop_read_status": [_p, C.POINTER(_i32)],
     "hop_clear_status": [_p],
+    "hop_build_is_checked": [],
     "hop_selftest_bounded_wait": [_p, _i32, _i32],
     "hop_level_stats": [_p, _i32, _p],
     "hop_timing_enable": [_p, _i32],
@@ -68,6 +70,10 @@ for _name, _args in SIGNATURES.items():
     _f = getattr(lib, _name)
     _f.argtypes = _args
     _f.restype = C.c_char_p if _name == "hop_last_error" else C.c_int
+
+
+def build_is_checked() -> bool:
+    return bool(lib.hop_build_is_checked())
 
 
 class DeviceSpan:
