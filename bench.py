@@ -263,6 +263,8 @@ def bench_config(args, cfg, env):
     steps = args.steps
     w = inputs.make_workload(cfg, P=args.P)
     w.stale_reduce = 1 if args.stale_reduce == "reuse" else 0
+    if args.momentum is not None:
+        w.momentum = args.momentum
     P_global = w.P
     lo, hi = shard_columns(P_global, world, rank)
     p0 = w.p0()[lo:hi].copy()
@@ -511,6 +513,7 @@ def main():
     ap.add_argument("--mix-kernel", type=int, default=0)
     ap.add_argument("--stale-reduce", default="new_only", choices=["new_only", "reuse"],
                     help="which updates inside the staleness bound enter a Reduce (default: Eq. 2 as printed)")
+    ap.add_argument("--momentum", type=float, default=None, help="override the configuration's momentum (a variant, not a headline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-secondary", action="store_true")

@@ -104,8 +104,9 @@ typedef enum hop_grad_mode {
     HOP_GRAD_SVM_CSR = 3     /* hinge-loss linear SVM, CSR rows (hop_bind_svm_csr)                 */
 } hop_grad_mode;
 
-/* AUTO: TENSOR for dense levels (>= 32 active workers consuming >= 32 updates each, N <= 128, P % 128 == 0, no
- * momentum or weight decay), else BULK (STAGED only when P % 4 != 0 and the level's tables exceed 32 KB of shared
+/* AUTO: TENSOR for dense levels (>= 32 active workers consuming >= 32 updates each, N <= 128, P % 128 == 0; with
+ * momentum or weight decay a pre-pass first turns G into the update direction in place, so a G the caller supplied
+ * is overwritten), else BULK (STAGED only when P % 4 != 0 and the level's tables exceed 32 KB of shared
  * memory).  hop_level_stats reports the kernel each level was planned with. */
 typedef enum hop_mix_kernel {
     HOP_MIX_AUTO = 0,

@@ -341,7 +341,8 @@ static int plan_level(hop_ctx* c, HopLevelHost& L, bool allow_tensor = true) {
     L.stage_rows = L.U + nG * (mom ? 2 : 1);
     int kernel = c->mix_kernel;
     // Tensor-core path: dense levels only (a contraction over <= 256 distinct slices for <= 128 workers).
-    const bool tc_ok = allow_tensor && c->g.N <= 128 && L.U <= 256 && L.nA > 0 && c->P % 128 == 0 && !mom && !decay &&
+    // (momentum and weight decay do not keep a level off it: the update direction is then formed in G by a pre-pass)
+    const bool tc_ok = allow_tensor && c->g.N <= 128 && L.U <= 256 && L.nA > 0 && c->P % 128 == 0 &&
                        (use_g || L.nG == 0 || c->serial) &&
                        hop_dense_tc_smem((L.U + 31) / 32 * 32) > 0;
     const bool dense = L.nA >= 32 && L.sumC >= 32 * (int64_t)L.nA;
@@ -577,6 +578,15 @@ static int run_level(hop_ctx* c, const HopLevelHost& L, const HopLevelDev& lv, c
     // None of the gradient kernels writes X or M, and each was launched with a full dependency on everything before it:
     // the mix may fetch its X and M rows while such a kernel drains (it waits before it reads G and before it stores).
     cfg.early_x = grad_kernel_in_front ? 1 : 0;
+    if (L.kernel == HOP_MIX_TENSOR && L.nG > 0 && cfg.use_g && (cfg.mu != 0.f || cfg.wd != 0.f)) {
+        // the dense path's epilogue applies -lr * G only: momentum and weight decay go into G first (cfg.mu / cfg.wd are
+        // already 0 here in the serial approach, where the apply kernel has done it all)
+        HOP_SPAN_BEGIN();
+        e = hop_launch_direction_dense(cfg, lv);
+        c->launches += 1;
+        if (e) HOP_FAIL(c, HOP_E_CUDA, std::string("update direction launch: ") + cudaGetErrorString((cudaError_t)e));
+        HOP_SPAN_END(2, 0);
+    }
     if (L.nA > 0) {
         HOP_SPAN_BEGIN();
         if (L.kernel == HOP_MIX_TENSOR)

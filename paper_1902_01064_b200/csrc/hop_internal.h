@@ -145,6 +145,8 @@ int hop_launch_svm_csr_apply(const HopLaunchCfg& c, const HopLevelDev& lv, const
                              const float* val, int32_t R, int32_t B, const float* coef, int32_t slot_shift);
 // serial approach, dense gradients: x_k <- x_k - lr * d in place for the level's NORMAL workers
 int hop_launch_apply_dense(const HopLaunchCfg& c, const HopLevelDev& lv);
+// dense (tensor-core) path with momentum or weight decay: G <- update direction, in place, before the mix
+int hop_launch_direction_dense(const HopLaunchCfg& c, const HopLevelDev& lv);
 bool hop_svm_dense_is_fused(int64_t P, int32_t B);   // the dense SVM gradient of a level is one launch instead of two
 int hop_checked_set_fence(const HopLaunchCfg& c);     // checked build only (no-op otherwise): bound-buffer ranges for the kernels
 bool hop_checked_build();

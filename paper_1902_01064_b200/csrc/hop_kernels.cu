@@ -876,6 +876,40 @@ apply_dense_kernel(float* __restrict__ X, float* __restrict__ M, const float* __
     }
 }
 
+// Update direction in place for the dense (tensor-core) path, whose epilogue applies -lr * G only: G <- g + lambda * x_k, through
+// the momentum buffer when there is one (m <- mu * m + G; G <- m), for the level's NORMAL workers.  One float4 per thread.
+template <bool MOMENTUM>
+__global__ void __launch_bounds__(256)
+direction_dense_kernel(const float* __restrict__ X, float* __restrict__ M, float* __restrict__ G, int64_t P, int S,
+                       float mu, float lam, HopLevelDev lv) {
+    const int worker = lv.grad_workers[blockIdx.y];
+    const int64_t c = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (c >= P) return;
+    const float* x = X + ((int64_t)worker * S + lv.level % S) * P + c;
+    float* g = G + (int64_t)worker * P + c;
+    float* m = MOMENTUM ? M + (int64_t)worker * P + c : nullptr;
+    const int n = (int)min((int64_t)4, P - c);
+    if (n == 4 && (P & 3) == 0) {
+        float4 gv = *reinterpret_cast<const float4*>(g);
+        if (lam != 0.f) {
+            const float4 xv = *reinterpret_cast<const float4*>(x);
+            gv.x = fmaf(lam, xv.x, gv.x); gv.y = fmaf(lam, xv.y, gv.y); gv.z = fmaf(lam, xv.z, gv.z); gv.w = fmaf(lam, xv.w, gv.w);
+        }
+        if constexpr (MOMENTUM) {
+            const float4 mv = *reinterpret_cast<const float4*>(m);
+            gv.x = fmaf(mu, mv.x, gv.x); gv.y = fmaf(mu, mv.y, gv.y); gv.z = fmaf(mu, mv.z, gv.z); gv.w = fmaf(mu, mv.w, gv.w);
+            *reinterpret_cast<float4*>(m) = gv;
+        }
+        *reinterpret_cast<float4*>(g) = gv;
+    } else {
+        for (int e = 0; e < n; ++e) {
+            float gv = lam != 0.f ? fmaf(lam, x[e], g[e]) : g[e];
+            if constexpr (MOMENTUM) { gv = fmaf(mu, m[e], gv); m[e] = gv; }
+            g[e] = gv;
+        }
+    }
+}
+
 constexpr int kStagedStages = 2;
 size_t staged_smem(const HopLaunchCfg& c, const HopLevelDev& lv) {
     const int nG = c.use_g ? lv.nG : 0;
@@ -1054,6 +1088,14 @@ int hop_launch_svm_csr_apply(const HopLaunchCfg& c, const HopLevelDev& lv, const
 
 int hop_launch_wait_selftest(int32_t* err_word, uint32_t polls, int32_t detail, void* stream) {
     wait_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(err_word, polls, detail);
+    return (int)cudaGetLastError();
+}
+
+int hop_launch_direction_dense(const HopLaunchCfg& c, const HopLevelDev& lv) {
+    if (lv.nG == 0) return 0;
+    dim3 grid((unsigned)(((c.P + 3) / 4 + 255) / 256), (unsigned)lv.nG);
+    if (c.mu != 0.f) direction_dense_kernel<true><<<grid, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.M, c.G, c.P, c.s + 1, c.mu, c.wd, lv);
+    else direction_dense_kernel<false><<<grid, 256, 0, (cudaStream_t)c.stream>>>(c.X, c.M, c.G, c.P, c.s + 1, c.mu, c.wd, lv);
     return (int)cudaGetLastError();
 }
 

@@ -628,8 +628,8 @@ def test_options_set_after_load_trace_plan_the_levels_again():
     assert max(np.abs(got[i] - want[i]).max() for i in range(w.N)) <= TOL_RUN * scale
     g.h.close()
     g = GpuRun(w, hop.MIX_TENSOR, x0=x0)
-    g.h.set_option(hop.OPT_WEIGHT_DECAY, 0.05)                 # the dense path has no weight decay: another kernel takes over
-    assert g.h.level_stats(2)["kernel"] == hop.MIX_BULK
+    g.h.set_option(hop.OPT_WEIGHT_DECAY, 0.05)                 # the dense path then forms the update direction in a pre-pass
+    assert g.h.level_stats(2)["kernel"] == hop.MIX_TENSOR
     got = g.run(w.iters)
     want, scale = _oracle_state(w, x0, w.iters, variant=dict(weight_decay=0.05))
     assert max(np.abs(got[i] - want[i]).max() for i in range(w.N)) <= TOL_RUN * scale
@@ -894,3 +894,17 @@ def test_full_size_graph_replay_equals_step_by_step(cfg):
             assert np.abs(got[i] - ref[i]).max() <= 1e-5 * (np.abs(ref[i]).max() + 1e-30)
         else:
             assert np.array_equal(got[i], ref[i])
+
+
+@pytest.mark.parametrize("momentum,variant", [(0.9, None), (0.0, dict(weight_decay=0.02)), (0.9, dict(weight_decay=0.02))])
+def test_tensor_path_with_momentum_and_weight_decay(momentum, variant):
+    # the dense path's epilogue applies -lr * G only: a pre-pass forms the update direction in G (momentum buffer, decay)
+    w = workload(5, P=1536, iters=10)
+    w.momentum = momentum
+    g = GpuRun(w, hop.MIX_TENSOR, variant=variant)
+    assert all(g.h.level_stats(k)["kernel"] == hop.MIX_TENSOR for k in range(w.iters))
+    g.h.close()
+    check(w, w.iters, TOL_RUN, hop.MIX_TENSOR, variant=variant)
+    check(w, 1, TOL_STEP, hop.MIX_TENSOR, perturb=True, variant=variant)
+    # and the general kernel gives the same within the run tolerance (both against the oracle)
+    check(w, w.iters, TOL_RUN, hop.MIX_BULK, perturb=True, variant=variant)
