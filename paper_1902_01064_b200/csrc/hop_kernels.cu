@@ -3,8 +3,10 @@
 //   mix_staged / mix_bulk   fused Recv-Reduce-Apply for one level: x_{k+1,i} = sum w * x_{v,j} - lr * d
 //                           (Fig. alg0 steps 2-3, Reduce of Fig. alg4 / Eq. 2), SGD or momentum, weight decay
 //   synth_grad              G[i][p] = sigma * normal(seed, i, k, p)
-//   svm_margin_* / svm_dense_grad / svm_csr_apply   hinge- or log-loss linear model gradient and sparse Apply
+//   svm_margin_* / svm_dense_grad / svm_dense_fused / svm_csr_apply   hinge- or log-loss linear model gradient and sparse Apply
 //   apply_dense             serial approach (Section 3.2): x_k <- x_k - lr * d before the level's Reduce
+//   direction_dense         G <- update direction (momentum, weight decay) ahead of the dense-graph kernel
+//   wait_selftest           a bounded wait that runs out, for the status-word path
 // (the dense-graph tensor-core kernel lives in hop_dense_tc.cu)
 //
 // In-place ring: version k+1 of a worker overwrites the slot of version k-s, which other workers may
